@@ -1,0 +1,171 @@
+/*
+ * svlm - the per-chunk KV-cache step of StreamingVLM-style streaming inference, for NVIDIA B200.
+ *
+ * One svlm_cache is the KV cache of one video stream.  Per one-second chunk the caller
+ *   1. appends the chunk's tokens (vision then text) with their native positions,
+ *   2. evicts (type-aware retention, left-shift of the retained positions, re-rotation of the
+ *      retained keys),
+ *   3. attends with the chunk's queries over the retained cache (chunk prefill),
+ *   4. and for every generated token appends one text token and attends with one query (decode).
+ *
+ * The operations follow Section 2.1 of the paper: the "Streaming-aware KV Cache" paragraph defines
+ * what is retained, the "Contiguous RoPE" paragraph defines the position re-indexing (1D and 3D).
+ *
+ * Conventions for every entry point
+ *   - returns SVLM_OK (0) or a negative svlm_status; never throws, never aborts the process;
+ *   - tensor arguments are DEVICE pointers owned by the caller unless the name ends in _host; the
+ *     library reads or writes them in the stream order of the cache's CUDA stream and keeps no
+ *     reference after the enqueued work has finished;
+ *   - work is enqueued on the cache's stream and the call returns without synchronising, except
+ *     svlm_cache_query, svlm_cache_status and the *_host variants' final copy where stated;
+ *   - conditions only the device can see (a type mix that overflows the capacity) set a sticky
+ *     status word that svlm_cache_status returns; the offending append is dropped as a whole;
+ *   - bf16 means the 16-bit brain-float bit pattern; Q/K are passed UN-rotated.
+ */
+#ifndef SVLM_H
+#define SVLM_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct svlm_cache svlm_cache; /* opaque; one per stream */
+
+enum svlm_token_type { SVLM_TEXT = 0, SVLM_VISION = 1 };
+enum svlm_rope_mode { SVLM_ROPE_1D = 0, SVLM_ROPE_MROPE = 1 };
+enum svlm_status {
+    SVLM_OK = 0,
+    SVLM_ERR_ARG = -1,      /* bad argument */
+    SVLM_ERR_CAPACITY = -2, /* append would exceed the capacity given at creation */
+    SVLM_ERR_ORDER = -3,    /* call sequence invalid (e.g. more queries than tokens appended) */
+    SVLM_ERR_CUDA = -4,     /* a CUDA runtime or driver call failed */
+    SVLM_ERR_TIMEOUT = -5,  /* a bounded device-side wait ran out */
+    SVLM_ERR_NOMEM = -6     /* device or host allocation failed */
+};
+
+/*
+ * Create the cache of one stream (paper Section 2.1, "Streaming-aware KV Cache": T_sink, V_window,
+ * T_window).  n_sink, vision_window and text_window are token counts (a 16 s vision window of
+ * 512 tokens/s is 8192).  capacity is the largest number of tokens that is ever stored at once,
+ * i.e. retained tokens plus everything appended before the next svlm_cache_evict.
+ * head_dim is 64 or 128.  Allocates device memory for `layers` K and V slabs
+ * ([layers][kv_heads][pages*128][head_dim] bf16, pages*128 >= capacity), per-token metadata and
+ * split-KV scratch; the current CUDA device at the time of the call owns the cache.
+ * Defaults: 1D RoPE with base 10000, sinks are text tokens, contiguous positions, legacy stream 0.
+ */
+int svlm_cache_create(svlm_cache** out, int layers, int kv_heads, int head_dim, int n_sink, int vision_window,
+                      int text_window, int capacity);
+
+/* Frees everything the cache owns after synchronising its stream.  Null is ignored. */
+void svlm_cache_destroy(svlm_cache* c);
+
+/*
+ * Rotary embedding geometry.  Pair (i, i + head_dim/2) rotates by position * base^(-2i/head_dim).
+ * SVLM_ROPE_1D: one position per token.  SVLM_ROPE_MROPE (3D positions of the Qwen-VL family,
+ * "Contiguous RoPE" paragraph): positions are (t,h,w) and sections[3] gives how many consecutive
+ * pairs use t, then h, then w; the three must sum to head_dim/2.  sections is ignored in 1D mode.
+ * Must be called before the first append.
+ */
+int svlm_cache_set_rope(svlm_cache* c, int mode, double base, const int sections[3]);
+
+/*
+ * Policy variants (defaults 0, 1).  sink_any_type != 0: the sinks are the first n_sink tokens of
+ * the stream whatever their type, instead of the first n_sink text tokens.  contiguous == 0:
+ * native RoPE, positions are never shifted (the paper's Table 4 ablation); eviction then only
+ * frees storage.  Must be called before the first append.
+ */
+int svlm_cache_set_policy(svlm_cache* c, int sink_any_type, int contiguous);
+
+/* CUDA stream (a cudaStream_t) on which all later work of this cache is enqueued. */
+int svlm_cache_set_stream(svlm_cache* c, void* cuda_stream);
+
+/*
+ * Append n tokens in stream order.
+ *   layer       -1: K and V are [layers][n][kv_heads][head_dim] and all layers are written;
+ *               l >= 0: K and V are [n][kv_heads][head_dim] for that layer only.
+ *   token_type  uint8 [n], SVLM_TEXT or SVLM_VISION    (read when layer is -1 or 0)
+ *   pos         int32 native positions, [n] in 1D mode or [n][3] = (t,h,w)   (read when layer is -1 or 0)
+ * The per-token metadata (stream ordinal, per-type ordinal, contiguous position = native position
+ * minus everything shifted so far, storage slot) is taken once per token, by the call with layer
+ * -1 or 0; calls for layers 1..layers-1 of the same tokens must follow with the same n and may pass
+ * null token_type/pos.  K is stored rotated at the token's contiguous position, V as is.
+ * Errors: SVLM_ERR_ARG; SVLM_ERR_CAPACITY when the host can already tell that n does not fit;
+ * otherwise an overflow is detected on the device, the append is dropped and the sticky status set.
+ */
+int svlm_cache_append(svlm_cache* c, int layer, const void* K, const void* V, const uint8_t* token_type,
+                      const int32_t* pos, int n);
+
+/*
+ * Evict, compact and re-index, all layers at once ("Streaming-aware KV Cache" and "Contiguous
+ * RoPE" paragraphs).  Keeps the n_sink sink tokens, the last text_window text tokens and the last
+ * vision_window vision tokens; every retained token's position moves left by the native position
+ * span of the evicted tokens before it, and its stored key is re-rotated by that amount; storage of
+ * evicted tokens is released.  Values never move.
+ */
+int svlm_cache_evict(svlm_cache* c);
+
+/*
+ * Grouped-query attention of the LAST n_q appended tokens over the stored tokens of one layer.
+ *   layer    l >= 0: Q and out are [n_q][q_heads][head_dim] bf16;
+ *            -1: all layers in one launch, Q and out are [layers][n_q][q_heads][head_dim].
+ *   q_pos    int32 native positions of the queries ([n_q] or [n_q][3])
+ * Query row r is the token with stream ordinal (tokens appended so far) - n_q + r; it is rotated at
+ * q_pos minus the total shift and sees every stored token whose ordinal does not exceed its own
+ * (retained history fully, the new chunk causally).  Query head h reads KV head
+ * h / (q_heads / kv_heads).  Scores are scaled by 1/sqrt(head_dim); a row that sees nothing yields
+ * zeros.  n_q == 1 takes the split-KV decode path, n_q >= 2 the chunk-prefill path.
+ * Errors: SVLM_ERR_ARG (q_heads not a multiple of kv_heads, n_q < 1, null pointers),
+ * SVLM_ERR_ORDER (n_q exceeds the tokens appended so far).
+ */
+int svlm_attend(svlm_cache* c, int layer, const void* Q, const int32_t* q_pos, int n_q, int q_heads, void* out);
+
+/*
+ * The same for n_caches independent streams in one launch (layer >= 0 only).  All caches must
+ * share geometry, RoPE settings, device and stream (the first cache's stream is used).
+ * Q and out are [n_caches][n_q][q_heads][head_dim]; q_pos is [n_caches][n_q] or [n_caches][n_q][3].
+ * n_caches <= 32.
+ */
+int svlm_attend_batched(svlm_cache* const* caches, int n_caches, int layer, const void* Q, const int32_t* q_pos,
+                        int n_q, int q_heads, void* out);
+
+/*
+ * Host-buffer variants: the same operations with K, V, token_type, pos / Q, q_pos, out in HOST
+ * memory (pinned memory makes the copies asynchronous).  The library stages them through device
+ * buffers it owns (grown on demand, which synchronises once).  svlm_attend_host returns after the
+ * result has arrived in out_host (it synchronises the stream).
+ */
+int svlm_cache_append_host(svlm_cache* c, int layer, const void* K_host, const void* V_host,
+                           const uint8_t* token_type_host, const int32_t* pos_host, int n);
+int svlm_attend_host(svlm_cache* c, int layer, const void* Q_host, const int32_t* q_pos_host, int n_q, int q_heads,
+                     void* out_host);
+
+/*
+ * Read back the stored tokens in stream order (HOST output buffers, each may be null; sized for
+ * `capacity` entries): stream ordinals, contiguous positions [n][3] (1D mode repeats the index),
+ * types.  n_kept and shift_total (sum of all left-shifts so far) are single values.
+ * Synchronises the cache's stream.
+ */
+int svlm_cache_query(svlm_cache* c, int64_t* n_kept, int64_t* gids, int32_t* pos, uint8_t* types, int64_t* shift_total);
+
+/*
+ * Copy the stored keys (as stored: rotated at the current positions) and values of one layer for
+ * the tokens svlm_cache_query lists, in that order, into HOST buffers [n_kept][kv_heads][head_dim]
+ * bf16 (either may be null).  Synchronises.  For tests and debugging.
+ */
+int svlm_cache_read_kv(svlm_cache* c, int layer, void* K_host, void* V_host);
+
+/* Sticky device-side status (SVLM_OK if nothing went wrong).  Synchronises the cache's stream. */
+int svlm_cache_status(svlm_cache* c);
+
+/* Number of kernels this library has launched in this process (all caches). */
+int64_t svlm_launch_count(void);
+
+/* Static description of a status code. */
+const char* svlm_strerror(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SVLM_H */

@@ -1,0 +1,134 @@
+// Key/value movement: writing appended tokens into their slots with the first rotation, and the
+// in-place re-rotation of retained keys after an eviction (paper Section 2.1, "Contiguous RoPE":
+// the indices of later tokens are shifted left; a stored key R(c)k becomes R(c-E)k = R(-E)R(c)k).
+// Both are streaming kernels: 16-byte accesses, no reuse, bound by HBM bandwidth.
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include "svlm_dev.h"
+#include "svlm_launch.h"
+
+namespace {
+
+struct __align__(16) Bf16x8 { __nv_bfloat162 v[4]; };
+
+// Rotate 8 consecutive pairs (lo[j], hi[j]) by (cs[j], sn[j]) in fp32, round to bf16.
+__device__ __forceinline__ void rotate8(Bf16x8& lo, Bf16x8& hi, const float* cs, const float* sn) {
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const float2 a = __bfloat1622float2(lo.v[j]);
+        const float2 b = __bfloat1622float2(hi.v[j]);
+        float2 ra, rb;
+        ra.x = a.x * cs[2 * j] - b.x * sn[2 * j];
+        rb.x = b.x * cs[2 * j] + a.x * sn[2 * j];
+        ra.y = a.y * cs[2 * j + 1] - b.y * sn[2 * j + 1];
+        rb.y = b.y * cs[2 * j + 1] + a.y * sn[2 * j + 1];
+        lo.v[j] = __float22bfloat162_rn(ra);
+        hi.v[j] = __float22bfloat162_rn(rb);
+    }
+}
+
+// One thread per (token, group of 8 pairs); it serves every kv head (and every layer when
+// layer < 0) of that token, so the sines are computed once.  Angles are formed in fp64.
+__global__ void __launch_bounds__(256) kv_write_kernel(SvlmCacheDev cd, int layer, const uint16_t* __restrict__ K,
+                                                       const uint16_t* __restrict__ V, int n) {
+    if (cd.ctrl->append_n != n) return;   // the metadata append was dropped (capacity) or does not match
+    const int half = cd.head_dim / 2;
+    const int groups = half / 8;          // threads per token
+    const int t = blockIdx.x * blockDim.x + threadIdx.x;
+    const int i = t / groups, g = t % groups;
+    if (i >= n) return;
+    const int slot = cd.new_slot[i];
+    float cs[8], sn[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const int pair = g * 8 + j;
+        const int axis = cd.rope_mode == 0 ? 0 : (pair < cd.sec_t ? 0 : (pair < cd.sec_th ? 1 : 2));
+        double s, c;
+        sincos((double)cd.new_c[3 * i + axis] * cd.theta[pair], &s, &c);
+        cs[j] = (float)c;
+        sn[j] = (float)s;
+    }
+    const int d = cd.head_dim;
+    const int l0 = layer < 0 ? 0 : layer, l1 = layer < 0 ? cd.layers : layer + 1;
+    for (int l = l0; l < l1; ++l) {
+        for (int h = 0; h < cd.kv_heads; ++h) {
+            const size_t src = (((size_t)(layer < 0 ? l : 0) * n + i) * cd.kv_heads + h) * d;
+            const size_t dst = (((size_t)l * cd.kv_heads + h) * cd.n_slots + slot) * d;
+            Bf16x8 lo = *reinterpret_cast<const Bf16x8*>(K + src + g * 8);
+            Bf16x8 hi = *reinterpret_cast<const Bf16x8*>(K + src + half + g * 8);
+            const uint4 vlo = *reinterpret_cast<const uint4*>(V + src + g * 8);
+            const uint4 vhi = *reinterpret_cast<const uint4*>(V + src + half + g * 8);
+            rotate8(lo, hi, cs, sn);
+            *reinterpret_cast<Bf16x8*>(cd.K + dst + g * 8) = lo;
+            *reinterpret_cast<Bf16x8*>(cd.K + dst + half + g * 8) = hi;
+            *reinterpret_cast<uint4*>(cd.V + dst + g * 8) = vlo;
+            *reinterpret_cast<uint4*>(cd.V + dst + half + g * 8) = vhi;
+        }
+    }
+}
+
+// Re-rotation after an eviction.  grid.x covers the slots, grid.y splits the layers.  A thread owns
+// (slot, group of 8 pairs) and walks its share of the [layer][kv_head] rows with the same sines;
+// the angle -E*theta is identical on the three MRoPE axes because all three indices of a token
+// shift by the same E.
+template <int UNROLL>
+__global__ void __launch_bounds__(256) evict_rotate_kernel(SvlmCacheDev cd, int layers_per_block) {
+    if (!cd.ctrl->evict_moved) return;
+    const int half = cd.head_dim / 2;
+    const int groups = half / 8;
+    const int t = blockIdx.x * blockDim.x + threadIdx.x;
+    const int slot = t / groups, g = t % groups;
+    if (slot >= cd.n_slots) return;
+    const int delta = cd.slot_delta[slot];
+    if (delta == 0) return;
+    float cs[8], sn[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        double s, c;
+        sincos(-(double)delta * cd.theta[g * 8 + j], &s, &c);
+        cs[j] = (float)c;
+        sn[j] = (float)s;
+    }
+    const int d = cd.head_dim;
+    const int row0 = blockIdx.y * layers_per_block * cd.kv_heads;
+    const int row1 = min(cd.layers, (blockIdx.y + 1) * layers_per_block) * cd.kv_heads;
+    const size_t stride = (size_t)cd.n_slots * d;
+    uint16_t* base = cd.K + (size_t)slot * d + g * 8;
+    for (int r = row0; r < row1; r += UNROLL) {
+        Bf16x8 lo[UNROLL], hi[UNROLL];
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u)
+            if (r + u < row1) {
+                lo[u] = *reinterpret_cast<const Bf16x8*>(base + (r + u) * stride);
+                hi[u] = *reinterpret_cast<const Bf16x8*>(base + (r + u) * stride + half);
+            }
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u)
+            if (r + u < row1) {
+                rotate8(lo[u], hi[u], cs, sn);
+                *reinterpret_cast<Bf16x8*>(base + (r + u) * stride) = lo[u];
+                *reinterpret_cast<Bf16x8*>(base + (r + u) * stride + half) = hi[u];
+            }
+    }
+}
+
+}  // namespace
+
+void svlm_launch_kv_write(const SvlmCacheDev& cd, int layer, const void* K, const void* V, int n, cudaStream_t st) {
+    const int groups = cd.head_dim / 16;
+    const int threads = n * groups;
+    kv_write_kernel<<<(threads + 255) / 256, 256, 0, st>>>(cd, layer, (const uint16_t*)K, (const uint16_t*)V, n);
+    svlm_count_launch();
+}
+
+void svlm_launch_evict_rotate(const SvlmCacheDev& cd, cudaStream_t st) {
+    const int groups = cd.head_dim / 16;
+    const int threads = cd.n_slots * groups;
+    // enough blocks in y to fill the machine a few times over, at least 4 rows per thread
+    int splits = 1;
+    while (splits < cd.layers && (cd.layers + splits - 1) / splits * cd.kv_heads > 8) ++splits;
+    const int lpb = (cd.layers + splits - 1) / splits;
+    dim3 grid((threads + 255) / 256, (cd.layers + lpb - 1) / lpb);
+    evict_rotate_kernel<4><<<grid, 256, 0, st>>>(cd, lpb);
+    svlm_count_launch();
+}

@@ -1,0 +1,20 @@
+// Host-side launchers of the kernels (one translation unit per kernel family).
+#pragma once
+#include <cuda_runtime.h>
+#include "svlm_dev.h"
+
+void svlm_count_launch();
+
+// metadata (svlm_meta.cu)
+void svlm_launch_append_meta(const SvlmCacheDev& cd, const unsigned char* types, const int* pos, int n, cudaStream_t st);
+void svlm_launch_evict_meta(const SvlmCacheDev& cd, cudaStream_t st);
+
+// key/value movement (svlm_kv.cu)
+// layer < 0: K,V are [layers][n][kv_heads][d]; otherwise [n][kv_heads][d] for that layer.
+void svlm_launch_kv_write(const SvlmCacheDev& cd, int layer, const void* K, const void* V, int n, cudaStream_t st);
+void svlm_launch_evict_rotate(const SvlmCacheDev& cd, cudaStream_t st);
+
+// attention (svlm_attend_simple.cu)
+// Q, out: [n_caches][n_layers][n_q][q_heads][d]; q_pos: [n_caches][n_q](x3)
+void svlm_launch_attend_simple(const SvlmAttendBatch& b, int layer0, int n_layers, const void* Q, const int* q_pos,
+                               int n_q, int q_heads, void* out, cudaStream_t st);

@@ -1,0 +1,382 @@
+// Metadata kernels: token bookkeeping on append, and the keep-mask / prefix-scan / re-index step
+// of eviction (paper Section 2.1, "Streaming-aware KV Cache" and "Contiguous RoPE").  Integer work
+// only; one CTA each (a few thousand records), results must be bit-exact.
+#include <cuda_runtime.h>
+#include "svlm_dev.h"
+#include "svlm_launch.h"
+
+namespace {
+
+constexpr int META_THREADS = 1024;
+constexpr int META_WARPS = META_THREADS / 32;
+
+// Block-wide exclusive scans over one value per thread.  `carry` is the running value over all
+// earlier rounds; on return every thread holds the exclusive result including the carry, and carry
+// has been advanced by this round's total.  All threads of the block must call.
+__device__ int block_excl_sum(int v, int& carry, int* warp_buf) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int inc = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        int t = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += t;
+    }
+    if (lane == 31) warp_buf[warp] = inc;
+    __syncthreads();
+    if (warp == 0) {
+        int w = warp_buf[lane];
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            int t = __shfl_up_sync(0xffffffffu, w, o);
+            if (lane >= o) w += t;
+        }
+        warp_buf[lane] = w;   // inclusive over warps
+    }
+    __syncthreads();
+    const int before = (warp ? warp_buf[warp - 1] : 0);
+    const int total = warp_buf[META_WARPS - 1];
+    const int res = carry + before + inc - v;
+    __syncthreads();
+    carry += total;
+    return res;
+}
+
+__device__ long long block_excl_sum64(long long v, long long& carry, long long* warp_buf) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    long long inc = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        long long t = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += t;
+    }
+    if (lane == 31) warp_buf[warp] = inc;
+    __syncthreads();
+    if (warp == 0) {
+        long long w = warp_buf[lane];
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            long long t = __shfl_up_sync(0xffffffffu, w, o);
+            if (lane >= o) w += t;
+        }
+        warp_buf[lane] = w;
+    }
+    __syncthreads();
+    const long long before = (warp ? warp_buf[warp - 1] : 0);
+    const long long total = warp_buf[META_WARPS - 1];
+    const long long res = carry + before + inc - v;
+    __syncthreads();
+    carry += total;
+    return res;
+}
+
+// Exclusive prefix maximum (carry = maximum over everything earlier).
+__device__ long long block_excl_max64(long long v, long long& carry, long long* warp_buf) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const long long NEG = -(1ll << 62);
+    long long inc = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        long long t = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc = max(inc, t);
+    }
+    long long exc = __shfl_up_sync(0xffffffffu, inc, 1);
+    if (lane == 0) exc = NEG;
+    if (lane == 31) warp_buf[warp] = inc;
+    __syncthreads();
+    if (warp == 0) {
+        long long w = warp_buf[lane];
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            long long t = __shfl_up_sync(0xffffffffu, w, o);
+            if (lane >= o) w = max(w, t);
+        }
+        warp_buf[lane] = w;
+    }
+    __syncthreads();
+    const long long before = (warp ? warp_buf[warp - 1] : NEG);
+    const long long total = warp_buf[META_WARPS - 1];
+    const long long res = max(carry, max(before, exc));
+    __syncthreads();
+    carry = max(carry, total);
+    return res;
+}
+
+__device__ __forceinline__ int ring_slot(const SvlmCacheDev& cd, int type, long long u) {
+    const int page = cd.page_table[type][(int)(u / SVLM_PAGE) & (cd.pt_size - 1)];
+    return page * SVLM_PAGE + (int)(u % SVLM_PAGE);
+}
+
+__device__ __forceinline__ long long ceil_page(long long x) { return (x + SVLM_PAGE - 1) / SVLM_PAGE; }
+
+// Rebuild the list of active pages (sink pages, then the text ring, then the vision ring).
+// Called by all threads after the slot metadata of this kernel has been written and synchronised.
+__device__ void rebuild_tiles(const SvlmCacheDev& cd, int sink_fill, const long long ring_lo[2],
+                              const long long ring_n[2]) {
+    const int n_sink_tiles = (sink_fill + SVLM_PAGE - 1) / SVLM_PAGE;
+    int cnt[2];
+    long long first[2];
+    for (int t = 0; t < 2; ++t) {
+        first[t] = ring_lo[t] / SVLM_PAGE;
+        cnt[t] = ring_n[t] > ring_lo[t] ? (int)((ring_n[t] - 1) / SVLM_PAGE - first[t] + 1) : 0;
+    }
+    const int total = n_sink_tiles + cnt[0] + cnt[1];
+    for (int i = threadIdx.x; i < total; i += blockDim.x) {
+        SvlmTile tl;
+        if (i < n_sink_tiles) {
+            tl.page = i;
+            tl.lo = 0;
+            tl.hi = min(SVLM_PAGE, sink_fill - i * SVLM_PAGE);
+        } else {
+            const int t = (i - n_sink_tiles < cnt[0]) ? 0 : 1;
+            const long long k = first[t] + (i - n_sink_tiles - (t ? cnt[0] : 0));
+            tl.page = cd.page_table[t][(int)k & (cd.pt_size - 1)];
+            tl.lo = (int)max(0ll, ring_lo[t] - k * SVLM_PAGE);
+            tl.hi = (int)min((long long)SVLM_PAGE, ring_n[t] - k * SVLM_PAGE);
+        }
+        tl.pad = 0;
+        tl.min_gid = cd.slot_gid[tl.page * SVLM_PAGE + tl.lo];
+        tl.max_gid = cd.slot_gid[tl.page * SVLM_PAGE + tl.hi - 1];
+        cd.tiles[i] = tl;
+    }
+    if (threadIdx.x == 0) cd.ctrl->n_tiles = total;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Append: stream ordinal, per-type ordinal, cursor advance a = max(0, max(p)+1 - cursor),
+// contiguous position c = p - shift_total, and the storage slot of each of the n new tokens.
+__global__ void __launch_bounds__(META_THREADS) append_meta_kernel(SvlmCacheDev cd, const unsigned char* types,
+                                                                   const int* pos, int n) {
+    __shared__ int wbuf[META_WARPS];
+    __shared__ long long wbuf64[META_WARPS];
+    __shared__ int s_cnt[3];     // text tokens; sink tokens of type TEXT / VISION in this append
+    __shared__ int s_ok;
+    SvlmCtrl* ctrl = cd.ctrl;
+    const int tid = threadIdx.x;
+    if (tid < 3) s_cnt[tid] = 0;
+    __syncthreads();
+
+    const long long n_total0 = ctrl->n_total;
+    const long long nt0[2] = {ctrl->n_type[0], ctrl->n_type[1]};
+    const long long cursor0 = ctrl->cursor;
+    const long long shift = cd.contiguous ? ctrl->shift_total : 0;
+    const long long ring_n0[2] = {ctrl->ring_n[0], ctrl->ring_n[1]};
+    const long long ring_lo0[2] = {ctrl->ring_lo[0], ctrl->ring_lo[1]};
+    const int sink_cnt0[2] = {ctrl->sink_cnt[0], ctrl->sink_cnt[1]};
+    const int sink_fill0 = ctrl->sink_fill;
+    const int n_stored0 = ctrl->n_stored;
+    const int free_top0 = ctrl->free_top;
+
+    // pass 0: totals
+    {
+        int text = 0, sink_text = 0, sink_vis = 0;
+        const long long any_limit = (long long)cd.n_sink - n_total0;   // tokens i < any_limit are sinks (any-type policy)
+        for (int i = tid; i < n; i += META_THREADS) {
+            const int ty = types[i] ? 1 : 0;
+            text += (ty == 0);
+            if (cd.sink_any && i < any_limit) { sink_text += (ty == 0); sink_vis += (ty == 1); }
+        }
+        atomicAdd(&s_cnt[0], text);
+        atomicAdd(&s_cnt[1], sink_text);
+        atomicAdd(&s_cnt[2], sink_vis);
+    }
+    __syncthreads();
+    const int n_text_new = s_cnt[0];
+    int sink_new[2];
+    if (cd.sink_any) {
+        sink_new[0] = s_cnt[1];
+        sink_new[1] = s_cnt[2];
+    } else {   // the first n_sink text ordinals are the sinks
+        long long room = (long long)cd.n_sink - nt0[0];
+        sink_new[0] = (int)max(0ll, min(room, (long long)n_text_new));
+        sink_new[1] = 0;
+    }
+    const int new_by_type[2] = {n_text_new, n - n_text_new};
+    long long ring_n1[2];
+    int pages_needed = 0;
+    for (int t = 0; t < 2; ++t) {
+        ring_n1[t] = ring_n0[t] + new_by_type[t] - sink_new[t];
+        pages_needed += (int)(ceil_page(ring_n1[t]) - ceil_page(ring_n0[t]));
+    }
+    if (tid == 0) {
+        const bool ok = (n_stored0 + n <= cd.capacity) && (pages_needed <= free_top0) &&
+                        (sink_fill0 + sink_new[0] + sink_new[1] <= cd.n_sink_pages * SVLM_PAGE);
+        s_ok = ok;
+        if (!ok) {
+            ctrl->append_n = 0;
+            if (ctrl->status == 0) ctrl->status = -2;   // SVLM_ERR_CAPACITY
+        } else {   // take pages for the ring ordinals this append opens
+            int top = free_top0;
+            for (int t = 0; t < 2; ++t)
+                for (long long k = ceil_page(ring_n0[t]); k < ceil_page(ring_n1[t]); ++k)
+                    cd.page_table[t][(int)k & (cd.pt_size - 1)] = cd.free_stack[--top];
+            ctrl->free_top = top;
+        }
+    }
+    __syncthreads();
+    if (!s_ok) return;
+
+    // pass 1: per-token scans, in rounds of one token per thread
+    int text_carry = 0;
+    long long top_carry = cursor0;
+    const int sink_final[2] = {sink_cnt0[0] + sink_new[0], sink_cnt0[1] + sink_new[1]};
+    for (int base = 0; base < n; base += META_THREADS) {
+        const int i = base + tid;
+        const bool live = i < n;
+        const int ty = live ? (types[i] ? 1 : 0) : 1;
+        long long p[3] = {0, 0, 0};
+        if (live) {
+            if (cd.rope_mode == 0) { p[0] = p[1] = p[2] = pos[i]; }
+            else { p[0] = pos[3 * i]; p[1] = pos[3 * i + 1]; p[2] = pos[3 * i + 2]; }
+        }
+        const long long top = live ? max(p[0], max(p[1], p[2])) + 1 : -(1ll << 62);
+        const int text_before = block_excl_sum(live && ty == 0, text_carry, wbuf);
+        const long long cur_before = block_excl_max64(top, top_carry, wbuf64);
+        if (!live) continue;
+        const long long gid = n_total0 + i;
+        const long long ord = nt0[ty] + (ty == 0 ? text_before : i - text_before);
+        const long long a = max(0ll, top - cur_before);
+        const bool is_sink = cd.sink_any ? (gid < cd.n_sink) : (ty == 0 && ord < cd.n_sink);
+        int slot;
+        if (is_sink) slot = (int)(cd.sink_any ? gid : ord);
+        else slot = ring_slot(cd, ty, ord - sink_final[ty]);
+        cd.slot_gid[slot] = gid;
+        cd.slot_type[slot] = (unsigned char)ty;
+        cd.slot_a[slot] = (int)a;
+        cd.slot_delta[slot] = 0;
+        cd.new_slot[i] = slot;
+        for (int k = 0; k < 3; ++k) {
+            const int c = (int)(p[k] - shift);
+            cd.slot_c[k * cd.n_slots + slot] = c;
+            cd.new_c[3 * i + k] = c;
+        }
+    }
+    __syncthreads();
+    const int sink_fill1 = sink_fill0 + sink_new[0] + sink_new[1];
+    rebuild_tiles(cd, sink_fill1, ring_lo0, ring_n1);
+    if (tid == 0) {
+        ctrl->n_total = n_total0 + n;
+        ctrl->n_type[0] = nt0[0] + new_by_type[0];
+        ctrl->n_type[1] = nt0[1] + new_by_type[1];
+        ctrl->cursor = top_carry;
+        ctrl->ring_n[0] = ring_n1[0];
+        ctrl->ring_n[1] = ring_n1[1];
+        ctrl->sink_cnt[0] = sink_final[0];
+        ctrl->sink_cnt[1] = sink_final[1];
+        ctrl->sink_fill = sink_fill1;
+        ctrl->n_stored = n_stored0 + n;
+        ctrl->append_n = n;
+    }
+}
+
+// Number of entries of the sorted list g[0..n) that are smaller than key.
+__device__ __forceinline__ int count_below(const long long* g, int n, long long key) {
+    int lo = 0, hi = n;
+    while (lo < hi) {
+        const int mid = (lo + hi) >> 1;
+        if (g[mid] < key) lo = mid + 1; else hi = mid;
+    }
+    return lo;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Evict: keep-mask (a suffix of each ring plus the sinks), prefix sums of the evicted tokens'
+// cursor advances, and the left-shift E(i) of every retained token i: the advances of all evicted
+// tokens that precede it in the stream.
+__global__ void __launch_bounds__(META_THREADS) evict_meta_kernel(SvlmCacheDev cd) {
+    __shared__ long long wbuf64[META_WARPS];
+    __shared__ int s_moved;
+    SvlmCtrl* ctrl = cd.ctrl;
+    const int tid = threadIdx.x;
+    if (tid == 0) s_moved = 0;
+
+    const long long ring_n[2] = {ctrl->ring_n[0], ctrl->ring_n[1]};
+    const long long lo0[2] = {ctrl->ring_lo[0], ctrl->ring_lo[1]};
+    const int sink_fill = ctrl->sink_fill;
+    const int win[2] = {cd.text_window, cd.vision_window};
+    long long lo1[2];
+    int n_ev[2];
+    for (int t = 0; t < 2; ++t) {
+        lo1[t] = min(ring_n[t], max(lo0[t], ring_n[t] - (long long)win[t]));
+        n_ev[t] = (int)(lo1[t] - lo0[t]);
+    }
+    __syncthreads();
+
+    // evicted tokens of each ring in ordinal (= stream) order, with exclusive prefix sums of a
+    long long freed[2];
+    for (int t = 0; t < 2; ++t) {
+        long long carry = 0;
+        for (int base = 0; base < n_ev[t]; base += META_THREADS) {
+            const int i = base + tid;
+            long long a = 0;
+            int slot = -1;
+            if (i < n_ev[t]) {
+                slot = ring_slot(cd, t, lo0[t] + i);
+                a = cd.contiguous ? cd.slot_a[slot] : 0;
+                cd.ev_gid[t][i] = cd.slot_gid[slot];
+            }
+            const long long ex = block_excl_sum64(a, carry, wbuf64);
+            if (i < n_ev[t]) {
+                cd.ev_pref[t][i] = ex;
+                cd.slot_gid[slot] = -1;
+                cd.slot_delta[slot] = 0;
+            }
+        }
+        freed[t] = carry;
+        if (tid == 0) cd.ev_pref[t][n_ev[t]] = carry;
+    }
+    __syncthreads();
+
+    // retained tokens: sinks, then the kept suffix of each ring
+    const long long kept_ring[2] = {ring_n[0] - lo1[0], ring_n[1] - lo1[1]};
+    const long long n_kept = sink_fill + kept_ring[0] + kept_ring[1];
+    int moved = 0;
+    for (long long i = tid; i < n_kept; i += META_THREADS) {
+        int slot;
+        if (i < sink_fill) slot = (int)i;
+        else if (i < sink_fill + kept_ring[0]) slot = ring_slot(cd, 0, lo1[0] + (i - sink_fill));
+        else slot = ring_slot(cd, 1, lo1[1] + (i - sink_fill - kept_ring[0]));
+        const long long g = cd.slot_gid[slot];
+        long long E = 0;
+        for (int t = 0; t < 2; ++t)
+            if (n_ev[t]) E += cd.ev_pref[t][count_below(cd.ev_gid[t], n_ev[t], g)];
+        cd.slot_delta[slot] = (int)E;
+        if (E) {
+            moved = 1;
+            for (int k = 0; k < 3; ++k) cd.slot_c[k * cd.n_slots + slot] -= (int)E;
+        }
+    }
+    if (moved) s_moved = 1;
+
+    // release pages that fell wholly below the new low-water mark
+    if (tid == 0) {
+        int top = ctrl->free_top;
+        for (int t = 0; t < 2; ++t) {
+            const long long end = min(lo1[t] / SVLM_PAGE, ceil_page(ring_n[t]));
+            for (long long k = lo0[t] / SVLM_PAGE; k < end; ++k)
+                cd.free_stack[top++] = cd.page_table[t][(int)k & (cd.pt_size - 1)];
+        }
+        ctrl->free_top = top;
+    }
+    __syncthreads();
+    rebuild_tiles(cd, sink_fill, lo1, ring_n);
+    if (tid == 0) {
+        ctrl->ring_lo[0] = lo1[0];
+        ctrl->ring_lo[1] = lo1[1];
+        ctrl->shift_total += freed[0] + freed[1];
+        ctrl->n_stored = (int)n_kept;
+        ctrl->evict_moved = s_moved;
+    }
+}
+
+}  // namespace
+
+void svlm_launch_append_meta(const SvlmCacheDev& cd, const unsigned char* types, const int* pos, int n,
+                             cudaStream_t st) {
+    append_meta_kernel<<<1, META_THREADS, 0, st>>>(cd, types, pos, n);
+    svlm_count_launch();
+}
+
+void svlm_launch_evict_meta(const SvlmCacheDev& cd, cudaStream_t st) {
+    evict_meta_kernel<<<1, META_THREADS, 0, st>>>(cd);
+    svlm_count_launch();
+}

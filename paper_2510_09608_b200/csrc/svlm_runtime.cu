@@ -1,0 +1,419 @@
+// Host runtime behind the C ABI of include/svlm.h: owns the device allocations of a cache,
+// validates arguments, and enqueues the kernels on the cache's stream.  No host synchronisation on
+// the hot path: everything the kernels need to know about the stream's state lives in the device
+// control block.
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <atomic>
+#include <cmath>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "../../include/svlm.h"
+#include "svlm_dev.h"
+#include "svlm_launch.h"
+
+static std::atomic<long long> g_launches{0};
+void svlm_count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
+
+struct svlm_cache {
+    SvlmCacheDev dev;
+    cudaStream_t stream = nullptr;
+    int device = 0;
+    std::vector<void*> allocs;
+    long long appended = 0;       // tokens accepted by the host checks so far
+    int pending_n = 0;            // n of the latest metadata append (layers 1.. must match)
+    bool configured_locked = false;
+    // staging for the *_host entry points
+    void* stage = nullptr;
+    size_t stage_bytes = 0;
+};
+
+namespace {
+
+#define SVLM_CUDA(call)                          \
+    do {                                         \
+        cudaError_t e_ = (call);                 \
+        if (e_ != cudaSuccess) return SVLM_ERR_CUDA; \
+    } while (0)
+
+struct DeviceGuard {
+    int prev = -1;
+    explicit DeviceGuard(int dev) {
+        cudaGetDevice(&prev);
+        if (prev != dev) cudaSetDevice(dev);
+        else prev = -1;
+    }
+    ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
+template <typename T>
+int dev_alloc(svlm_cache* c, T** p, size_t count, bool zero = true) {
+    void* q = nullptr;
+    if (cudaMalloc(&q, std::max<size_t>(count, 1) * sizeof(T)) != cudaSuccess) return SVLM_ERR_NOMEM;
+    c->allocs.push_back(q);
+    if (zero && cudaMemset(q, 0, std::max<size_t>(count, 1) * sizeof(T)) != cudaSuccess) return SVLM_ERR_CUDA;
+    *p = static_cast<T*>(q);
+    return SVLM_OK;
+}
+
+void fill_theta(SvlmCacheDev& d, double base) {
+    for (int i = 0; i < d.head_dim / 2; ++i) d.theta[i] = std::pow(base, -2.0 * i / d.head_dim);
+}
+
+int ensure_stage(svlm_cache* c, size_t bytes) {
+    if (bytes <= c->stage_bytes) return SVLM_OK;
+    SVLM_CUDA(cudaStreamSynchronize(c->stream));
+    if (c->stage) cudaFree(c->stage);
+    c->stage = nullptr;
+    c->stage_bytes = 0;
+    if (cudaMalloc(&c->stage, bytes) != cudaSuccess) return SVLM_ERR_NOMEM;
+    c->stage_bytes = bytes;
+    return SVLM_OK;
+}
+
+void fill_view(const svlm_cache* c, SvlmAttendView& v) {
+    v.K = c->dev.K;
+    v.V = c->dev.V;
+    v.ctrl = c->dev.ctrl;
+    v.tiles = c->dev.tiles;
+    v.slot_gid = c->dev.slot_gid;
+    v.ws = c->dev.ws;
+}
+
+void fill_batch_geometry(const svlm_cache* c, SvlmAttendBatch& b) {
+    b.layers = c->dev.layers;
+    b.kv_heads = c->dev.kv_heads;
+    b.head_dim = c->dev.head_dim;
+    b.n_slots = c->dev.n_slots;
+    b.rope_mode = c->dev.rope_mode;
+    b.sec_t = c->dev.sec_t;
+    b.sec_th = c->dev.sec_th;
+    std::memcpy(b.theta, c->dev.theta, sizeof b.theta);
+}
+
+int attend_common(svlm_cache* const* caches, int n_caches, int layer, const void* Q, const int32_t* q_pos, int n_q,
+                  int q_heads, void* out) {
+    svlm_cache* c0 = caches[0];
+    if (!Q || !q_pos || !out || n_q < 1 || q_heads < 1) return SVLM_ERR_ARG;
+    if (q_heads % c0->dev.kv_heads) return SVLM_ERR_ARG;
+    if (layer < -1 || layer >= c0->dev.layers) return SVLM_ERR_ARG;
+    SvlmAttendBatch b;
+    b.n_caches = n_caches;
+    fill_batch_geometry(c0, b);
+    for (int i = 0; i < n_caches; ++i) {
+        const svlm_cache* c = caches[i];
+        if (!c) return SVLM_ERR_ARG;
+        if (c->dev.layers != c0->dev.layers || c->dev.kv_heads != c0->dev.kv_heads ||
+            c->dev.head_dim != c0->dev.head_dim || c->dev.n_slots != c0->dev.n_slots ||
+            c->dev.rope_mode != c0->dev.rope_mode || c->dev.sec_t != c0->dev.sec_t || c->dev.sec_th != c0->dev.sec_th ||
+            c->dev.theta[1] != c0->dev.theta[1] || c->device != c0->device)
+            return SVLM_ERR_ARG;
+        if (n_q > c->appended) return SVLM_ERR_ORDER;
+        fill_view(c, b.view[i]);
+    }
+    DeviceGuard guard(c0->device);
+    const int layer0 = layer < 0 ? 0 : layer;
+    const int n_layers = layer < 0 ? c0->dev.layers : 1;
+    svlm_launch_attend_simple(b, layer0, n_layers, Q, q_pos, n_q, q_heads, out, c0->stream);
+    SVLM_CUDA(cudaGetLastError());
+    return SVLM_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int svlm_cache_create(svlm_cache** out, int layers, int kv_heads, int head_dim, int n_sink, int vision_window,
+                      int text_window, int capacity) {
+    if (!out) return SVLM_ERR_ARG;
+    *out = nullptr;
+    if (layers < 1 || kv_heads < 1 || (head_dim != 64 && head_dim != 128) || n_sink < 0 || vision_window < 0 ||
+        text_window < 0 || capacity < 1)
+        return SVLM_ERR_ARG;
+    svlm_cache* c = new (std::nothrow) svlm_cache;
+    if (!c) return SVLM_ERR_NOMEM;
+    if (cudaGetDevice(&c->device) != cudaSuccess) { delete c; return SVLM_ERR_CUDA; }
+    SvlmCacheDev& d = c->dev;
+    std::memset(&d, 0, sizeof d);
+    d.layers = layers; d.kv_heads = kv_heads; d.head_dim = head_dim;
+    d.n_sink = n_sink; d.vision_window = vision_window; d.text_window = text_window; d.capacity = capacity;
+    d.n_sink_pages = (std::min(n_sink, capacity) + SVLM_PAGE - 1) / SVLM_PAGE;
+    // two rings, each with at most one partial page at either end
+    d.n_pages = d.n_sink_pages + (capacity + SVLM_PAGE - 1) / SVLM_PAGE + 4;
+    d.n_slots = d.n_pages * SVLM_PAGE;
+    d.pt_size = 1;
+    while (d.pt_size <= d.n_pages) d.pt_size <<= 1;
+    d.rope_mode = SVLM_ROPE_1D; d.sink_any = 0; d.contiguous = 1;
+    d.sec_t = d.sec_th = head_dim / 2;
+    fill_theta(d, 10000.0);
+
+    int rc = SVLM_OK;
+    const size_t slab = (size_t)layers * kv_heads * d.n_slots * head_dim;
+    auto A = [&](int r) { if (rc == SVLM_OK) rc = r; };
+    A(dev_alloc(c, &d.ctrl, 1));
+    A(dev_alloc(c, &d.free_stack, d.n_pages));
+    A(dev_alloc(c, &d.page_table[0], d.pt_size));
+    A(dev_alloc(c, &d.page_table[1], d.pt_size));
+    A(dev_alloc(c, &d.slot_gid, d.n_slots));
+    A(dev_alloc(c, &d.slot_c, 3 * (size_t)d.n_slots));
+    A(dev_alloc(c, &d.slot_a, d.n_slots));
+    A(dev_alloc(c, &d.slot_delta, d.n_slots));
+    A(dev_alloc(c, &d.slot_type, d.n_slots));
+    A(dev_alloc(c, &d.tiles, d.n_pages));
+    A(dev_alloc(c, &d.new_slot, capacity));
+    A(dev_alloc(c, &d.new_c, 3 * (size_t)capacity));
+    for (int t = 0; t < 2; ++t) {
+        A(dev_alloc(c, &d.ev_gid[t], capacity));
+        A(dev_alloc(c, &d.ev_pref[t], (size_t)capacity + 1));
+    }
+    A(dev_alloc(c, &d.K, slab));
+    A(dev_alloc(c, &d.V, slab));
+    if (rc == SVLM_OK) {
+        // pool pages on the free stack (top of the stack = lowest page number)
+        std::vector<int> stack;
+        for (int p = d.n_pages - 1; p >= d.n_sink_pages; --p) stack.push_back(p);
+        SvlmCtrl ctrl;
+        std::memset(&ctrl, 0, sizeof ctrl);
+        ctrl.free_top = (int)stack.size();
+        std::vector<long long> minus1(d.n_slots, -1);
+        if (cudaMemcpy(d.free_stack, stack.data(), stack.size() * sizeof(int), cudaMemcpyHostToDevice) != cudaSuccess ||
+            cudaMemcpy(d.ctrl, &ctrl, sizeof ctrl, cudaMemcpyHostToDevice) != cudaSuccess ||
+            cudaMemcpy(d.slot_gid, minus1.data(), minus1.size() * sizeof(long long), cudaMemcpyHostToDevice) !=
+                cudaSuccess)
+            rc = SVLM_ERR_CUDA;
+    }
+    if (rc != SVLM_OK) {
+        for (void* p : c->allocs) cudaFree(p);
+        delete c;
+        return rc;
+    }
+    *out = c;
+    return SVLM_OK;
+}
+
+void svlm_cache_destroy(svlm_cache* c) {
+    if (!c) return;
+    DeviceGuard guard(c->device);
+    cudaStreamSynchronize(c->stream);
+    for (void* p : c->allocs) cudaFree(p);
+    if (c->stage) cudaFree(c->stage);
+    delete c;
+}
+
+int svlm_cache_set_rope(svlm_cache* c, int mode, double base, const int sections[3]) {
+    if (!c || !(base > 1.0) || (mode != SVLM_ROPE_1D && mode != SVLM_ROPE_MROPE)) return SVLM_ERR_ARG;
+    if (c->configured_locked) return SVLM_ERR_ORDER;
+    const int half = c->dev.head_dim / 2;
+    if (mode == SVLM_ROPE_MROPE) {
+        if (!sections || sections[0] < 0 || sections[1] < 0 || sections[2] < 0 ||
+            sections[0] + sections[1] + sections[2] != half)
+            return SVLM_ERR_ARG;
+        c->dev.sec_t = sections[0];
+        c->dev.sec_th = sections[0] + sections[1];
+    } else {
+        c->dev.sec_t = c->dev.sec_th = half;
+    }
+    c->dev.rope_mode = mode;
+    fill_theta(c->dev, base);
+    return SVLM_OK;
+}
+
+int svlm_cache_set_policy(svlm_cache* c, int sink_any_type, int contiguous) {
+    if (!c) return SVLM_ERR_ARG;
+    if (c->configured_locked) return SVLM_ERR_ORDER;
+    c->dev.sink_any = sink_any_type ? 1 : 0;
+    c->dev.contiguous = contiguous ? 1 : 0;
+    return SVLM_OK;
+}
+
+int svlm_cache_set_stream(svlm_cache* c, void* cuda_stream) {
+    if (!c) return SVLM_ERR_ARG;
+    c->stream = static_cast<cudaStream_t>(cuda_stream);
+    return SVLM_OK;
+}
+
+int svlm_cache_append(svlm_cache* c, int layer, const void* K, const void* V, const uint8_t* token_type,
+                      const int32_t* pos, int n) {
+    if (!c || !K || !V || n < 1 || layer < -1 || layer >= c->dev.layers) return SVLM_ERR_ARG;
+    DeviceGuard guard(c->device);
+    if (layer <= 0) {
+        if (!token_type || !pos) return SVLM_ERR_ARG;
+        if (n > c->dev.capacity) return SVLM_ERR_CAPACITY;
+        c->configured_locked = true;
+        svlm_launch_append_meta(c->dev, token_type, pos, n, c->stream);
+        c->appended += n;
+        c->pending_n = n;
+    } else if (n != c->pending_n) {
+        return SVLM_ERR_ORDER;
+    }
+    svlm_launch_kv_write(c->dev, layer, K, V, n, c->stream);
+    SVLM_CUDA(cudaGetLastError());
+    return SVLM_OK;
+}
+
+int svlm_cache_evict(svlm_cache* c) {
+    if (!c) return SVLM_ERR_ARG;
+    DeviceGuard guard(c->device);
+    svlm_launch_evict_meta(c->dev, c->stream);
+    if (c->dev.contiguous) svlm_launch_evict_rotate(c->dev, c->stream);
+    SVLM_CUDA(cudaGetLastError());
+    return SVLM_OK;
+}
+
+int svlm_attend(svlm_cache* c, int layer, const void* Q, const int32_t* q_pos, int n_q, int q_heads, void* out) {
+    if (!c) return SVLM_ERR_ARG;
+    svlm_cache* one[1] = {c};
+    return attend_common(one, 1, layer, Q, q_pos, n_q, q_heads, out);
+}
+
+int svlm_attend_batched(svlm_cache* const* caches, int n_caches, int layer, const void* Q, const int32_t* q_pos,
+                        int n_q, int q_heads, void* out) {
+    if (!caches || n_caches < 1 || n_caches > SVLM_MAX_BATCH || layer < 0) return SVLM_ERR_ARG;
+    if (!caches[0]) return SVLM_ERR_ARG;
+    return attend_common(caches, n_caches, layer, Q, q_pos, n_q, q_heads, out);
+}
+
+int svlm_cache_append_host(svlm_cache* c, int layer, const void* K_host, const void* V_host,
+                           const uint8_t* token_type_host, const int32_t* pos_host, int n) {
+    if (!c || !K_host || !V_host || n < 1 || layer < -1 || layer >= c->dev.layers) return SVLM_ERR_ARG;
+    if (layer <= 0 && (!token_type_host || !pos_host)) return SVLM_ERR_ARG;
+    DeviceGuard guard(c->device);
+    const int nl = layer < 0 ? c->dev.layers : 1;
+    const size_t kv_bytes = (size_t)nl * n * c->dev.kv_heads * c->dev.head_dim * 2;
+    const size_t pos_bytes = (size_t)n * (c->dev.rope_mode == SVLM_ROPE_1D ? 1 : 3) * sizeof(int32_t);
+    const size_t ty_off = 2 * kv_bytes, pos_off = (ty_off + n + 255) / 256 * 256;
+    int rc = ensure_stage(c, pos_off + pos_bytes);
+    if (rc != SVLM_OK) return rc;
+    char* s = static_cast<char*>(c->stage);
+    SVLM_CUDA(cudaMemcpyAsync(s, K_host, kv_bytes, cudaMemcpyHostToDevice, c->stream));
+    SVLM_CUDA(cudaMemcpyAsync(s + kv_bytes, V_host, kv_bytes, cudaMemcpyHostToDevice, c->stream));
+    if (layer <= 0) {
+        SVLM_CUDA(cudaMemcpyAsync(s + ty_off, token_type_host, n, cudaMemcpyHostToDevice, c->stream));
+        SVLM_CUDA(cudaMemcpyAsync(s + pos_off, pos_host, pos_bytes, cudaMemcpyHostToDevice, c->stream));
+    }
+    return svlm_cache_append(c, layer, s, s + kv_bytes, reinterpret_cast<const uint8_t*>(s + ty_off),
+                             reinterpret_cast<const int32_t*>(s + pos_off), n);
+}
+
+int svlm_attend_host(svlm_cache* c, int layer, const void* Q_host, const int32_t* q_pos_host, int n_q, int q_heads,
+                     void* out_host) {
+    if (!c || !Q_host || !q_pos_host || !out_host || n_q < 1 || q_heads < 1 || layer < -1 || layer >= c->dev.layers)
+        return SVLM_ERR_ARG;
+    DeviceGuard guard(c->device);
+    const int nl = layer < 0 ? c->dev.layers : 1;
+    const size_t q_bytes = ((size_t)nl * n_q * q_heads * c->dev.head_dim * 2 + 255) / 256 * 256;
+    const size_t pos_bytes = ((size_t)n_q * (c->dev.rope_mode == SVLM_ROPE_1D ? 1 : 3) * sizeof(int32_t) + 255) / 256 * 256;
+    int rc = ensure_stage(c, 2 * q_bytes + pos_bytes);
+    if (rc != SVLM_OK) return rc;
+    char* s = static_cast<char*>(c->stage);
+    SVLM_CUDA(cudaMemcpyAsync(s, Q_host, (size_t)nl * n_q * q_heads * c->dev.head_dim * 2, cudaMemcpyHostToDevice,
+                              c->stream));
+    SVLM_CUDA(cudaMemcpyAsync(s + 2 * q_bytes, q_pos_host,
+                              (size_t)n_q * (c->dev.rope_mode == SVLM_ROPE_1D ? 1 : 3) * sizeof(int32_t),
+                              cudaMemcpyHostToDevice, c->stream));
+    rc = svlm_attend(c, layer, s, reinterpret_cast<const int32_t*>(s + 2 * q_bytes), n_q, q_heads, s + q_bytes);
+    if (rc != SVLM_OK) return rc;
+    SVLM_CUDA(cudaMemcpyAsync(out_host, s + q_bytes, (size_t)nl * n_q * q_heads * c->dev.head_dim * 2,
+                              cudaMemcpyDeviceToHost, c->stream));
+    SVLM_CUDA(cudaStreamSynchronize(c->stream));
+    return SVLM_OK;
+}
+
+// Host mirror of the stored tokens in stream order: (gid, slot) pairs sorted by gid.
+static int snapshot(svlm_cache* c, std::vector<std::pair<long long, int>>& order, SvlmCtrl& ctrl) {
+    const SvlmCacheDev& d = c->dev;
+    SVLM_CUDA(cudaStreamSynchronize(c->stream));
+    SVLM_CUDA(cudaMemcpy(&ctrl, d.ctrl, sizeof ctrl, cudaMemcpyDeviceToHost));
+    std::vector<SvlmTile> tiles(std::max(ctrl.n_tiles, 1));
+    std::vector<long long> gid(d.n_slots);
+    SVLM_CUDA(cudaMemcpy(tiles.data(), d.tiles, ctrl.n_tiles * sizeof(SvlmTile), cudaMemcpyDeviceToHost));
+    SVLM_CUDA(cudaMemcpy(gid.data(), d.slot_gid, gid.size() * sizeof(long long), cudaMemcpyDeviceToHost));
+    order.clear();
+    for (int t = 0; t < ctrl.n_tiles; ++t)
+        for (int o = tiles[t].lo; o < tiles[t].hi; ++o) {
+            const int slot = tiles[t].page * SVLM_PAGE + o;
+            order.emplace_back(gid[slot], slot);
+        }
+    std::sort(order.begin(), order.end());
+    return SVLM_OK;
+}
+
+int svlm_cache_query(svlm_cache* c, int64_t* n_kept, int64_t* gids, int32_t* pos, uint8_t* types,
+                     int64_t* shift_total) {
+    if (!c) return SVLM_ERR_ARG;
+    DeviceGuard guard(c->device);
+    const SvlmCacheDev& d = c->dev;
+    std::vector<std::pair<long long, int>> order;
+    SvlmCtrl ctrl;
+    int rc = snapshot(c, order, ctrl);
+    if (rc != SVLM_OK) return rc;
+    std::vector<int> cpos(3 * (size_t)d.n_slots);
+    std::vector<unsigned char> ty(d.n_slots);
+    SVLM_CUDA(cudaMemcpy(cpos.data(), d.slot_c, cpos.size() * sizeof(int), cudaMemcpyDeviceToHost));
+    SVLM_CUDA(cudaMemcpy(ty.data(), d.slot_type, ty.size(), cudaMemcpyDeviceToHost));
+    if ((long long)order.size() != ctrl.n_stored) return SVLM_ERR_CUDA;   // tile list and count disagree
+    for (size_t i = 0; i < order.size(); ++i) {
+        const int slot = order[i].second;
+        if (gids) gids[i] = order[i].first;
+        if (types) types[i] = ty[slot];
+        if (pos) for (int k = 0; k < 3; ++k) pos[3 * i + k] = cpos[(size_t)k * d.n_slots + slot];
+    }
+    if (n_kept) *n_kept = (int64_t)order.size();
+    if (shift_total) *shift_total = ctrl.shift_total;
+    return SVLM_OK;
+}
+
+int svlm_cache_read_kv(svlm_cache* c, int layer, void* K_host, void* V_host) {
+    if (!c || layer < 0 || layer >= c->dev.layers) return SVLM_ERR_ARG;
+    DeviceGuard guard(c->device);
+    const SvlmCacheDev& d = c->dev;
+    std::vector<std::pair<long long, int>> order;
+    SvlmCtrl ctrl;
+    int rc = snapshot(c, order, ctrl);
+    if (rc != SVLM_OK) return rc;
+    const size_t per_layer = (size_t)d.kv_heads * d.n_slots * d.head_dim;
+    std::vector<uint16_t> slab(per_layer);
+    for (int which = 0; which < 2; ++which) {
+        uint16_t* dst = static_cast<uint16_t*>(which ? V_host : K_host);
+        if (!dst) continue;
+        const uint16_t* src = (which ? d.V : d.K) + (size_t)layer * per_layer;
+        SVLM_CUDA(cudaMemcpy(slab.data(), src, per_layer * sizeof(uint16_t), cudaMemcpyDeviceToHost));
+        for (size_t i = 0; i < order.size(); ++i)
+            for (int h = 0; h < d.kv_heads; ++h)
+                std::memcpy(dst + (i * d.kv_heads + h) * d.head_dim,
+                            slab.data() + ((size_t)h * d.n_slots + order[i].second) * d.head_dim,
+                            d.head_dim * sizeof(uint16_t));
+    }
+    return SVLM_OK;
+}
+
+int svlm_cache_status(svlm_cache* c) {
+    if (!c) return SVLM_ERR_ARG;
+    DeviceGuard guard(c->device);
+    SVLM_CUDA(cudaStreamSynchronize(c->stream));
+    SvlmCtrl ctrl;
+    SVLM_CUDA(cudaMemcpy(&ctrl, c->dev.ctrl, sizeof ctrl, cudaMemcpyDeviceToHost));
+    return ctrl.status;
+}
+
+int64_t svlm_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+const char* svlm_strerror(int status) {
+    switch (status) {
+        case SVLM_OK: return "ok";
+        case SVLM_ERR_ARG: return "bad argument";
+        case SVLM_ERR_CAPACITY: return "cache capacity exceeded";
+        case SVLM_ERR_ORDER: return "call out of order";
+        case SVLM_ERR_CUDA: return "CUDA call failed";
+        case SVLM_ERR_TIMEOUT: return "bounded device wait ran out";
+        case SVLM_ERR_NOMEM: return "out of memory";
+        default: return "unknown status";
+    }
+}
+
+}  // extern "C"

@@ -1,0 +1,128 @@
+"""GPU parity: the CUDA library against the CPU checker, through the C ABI, on seeded streams."""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+pytestmark = pytest.mark.gpu
+
+
+def _wl(n):
+    from paper_2510_09608_b200 import streamgen as sg
+    return sg.workloads()[n]
+
+
+def test_config1_every_output():
+    """Workload 1: the whole 20-chunk stream; every kept index, position, key and output is compared."""
+    from harness import SideBySide, assert_close
+    wl = _wl(1)
+    s = SideBySide(wl)
+    worst = [0.0, 0.0]
+    for chunk in range(wl.chunks):
+        s.append_chunk()
+        s.evict()
+        n = s.check_metadata()
+        assert n <= wl.retained
+        s.check_kv(0)
+        st = s.attend(0)
+        assert_close(st)
+        worst = [max(worst[0], st[0]), max(worst[1], st[1])]
+        for _ in range(wl.decode_steps):
+            s.append_decode_token()
+            assert_close(s.attend(0))
+        s.check_metadata()
+    print("config 1 worst max/mean abs error", worst)
+
+
+@pytest.mark.parametrize("sink_any,contiguous", [(False, True), (True, True), (False, False)])
+def test_scaled_mrope_stream_multi_layer(sink_any, contiguous):
+    """A shrunk workload-2 shape (MRoPE, GQA 28/4, d=128, 3 layers) that crosses several pages,
+    partial pages and a ragged tail; every chunk fully compared, per-layer and all-layer calls."""
+    from harness import SideBySide, assert_close
+    wl = dataclasses.replace(_wl(2), layers=3, n_sink=40, vision_window=3 * 128, text_window=70,
+                             frames=2, grid_h=8, grid_w=8, text_max=24, decode_steps=3)
+    s = SideBySide(wl, sink_any=sink_any, contiguous=contiguous)
+    for chunk in range(12):
+        s.append_chunk(per_layer_calls=(chunk % 2 == 1))
+        s.evict()
+        s.check_metadata()
+        layer = chunk % 3
+        s.check_kv(layer)
+        assert_close(s.attend(layer, all_layers=(chunk % 3 == 0)))
+        for _ in range(wl.decode_steps):
+            s.append_decode_token()
+            assert_close(s.attend((layer + 1) % 3))
+    s.evict()
+    s.evict()      # a second evict with nothing new must change nothing
+    s.check_metadata()
+    s.check_kv(1)
+
+
+@pytest.mark.parametrize("S,Vw,Tw", [(0, 64, 16), (8, 0, 16), (8, 64, 0), (0, 0, 0), (300, 64, 16)])
+def test_degenerate_policies(S, Vw, Tw):
+    """Window and sink sizes of zero (the paper's ablation grid has 0-sized sinks and windows), and
+    sinks spanning several pages."""
+    from harness import SideBySide, assert_close
+    wl = dataclasses.replace(_wl(1), n_sink=S, vision_window=Vw, text_window=Tw, text_max=30)
+    s = SideBySide(wl, capacity=512)
+    for chunk in range(14):
+        s.append_chunk()
+        s.evict()
+        s.check_metadata()
+        s.check_kv(0)
+        st = s.attend(0)
+        assert_close(st)
+        s.append_decode_token()
+        assert_close(s.attend(0))
+
+
+def test_batched_streams_match_single_calls():
+    from harness import SideBySide, bits_to_dev, dev_to_f64
+    from paper_2510_09608_b200 import binding
+    wl = dataclasses.replace(_wl(2), n_sink=16, vision_window=256, text_window=32, frames=1, grid_h=8, grid_w=8)
+    sides = [SideBySide(wl, stream=i) for i in range(3)]
+    for s in sides:
+        for _ in range(4 + sides.index(s)):
+            s.append_chunk()
+            s.evict()
+        s.append_decode_token()
+    Q = np.stack([s.stream.q(0, s.last[0]) for s in sides])
+    qpos = torch.from_numpy(np.stack([s.last[2] for s in sides])).cuda()
+    out = dev_to_f64(binding.attend_batched([s.cache for s in sides], 0, bits_to_dev(Q), qpos))
+    for i, s in enumerate(sides):
+        s._give_values_to_ref(0)
+        want = s.ref.attend(0, Q[i], s.last[2])
+        err = np.abs(out[i] - want)
+        assert err.max() <= 1e-2 and err.mean() <= 1e-3
+
+
+def test_errors_and_capacity():
+    from paper_2510_09608_b200 import binding
+    with pytest.raises(binding.SvlmError):
+        binding.Cache(1, 1, 96, 4, 8, 8, 64)          # head_dim must be 64 or 128
+    c = binding.Cache(1, 1, 64, 4, 8, 8, 64)
+    K = torch.zeros(40, 1, 64, dtype=torch.bfloat16, device="cuda")
+    ty = torch.zeros(40, dtype=torch.uint8, device="cuda")
+    pos = torch.arange(40, dtype=torch.int32, device="cuda")
+    with pytest.raises(binding.SvlmError) as e:
+        c.attend(0, K[:1], pos[:1])
+    assert e.value.status == binding.ERR_ORDER           # nothing appended yet
+    c.append(0, K, K, ty, pos)
+    c2 = binding.Cache(1, 2, 64, 4, 8, 8, 64)
+    c2.append(0, torch.zeros(4, 2, 64, dtype=torch.bfloat16, device="cuda"),
+              torch.zeros(4, 2, 64, dtype=torch.bfloat16, device="cuda"), ty[:4], pos[:4])
+    with pytest.raises(binding.SvlmError) as e:          # 3 query heads over 2 kv heads
+        c2.attend(0, torch.zeros(1, 3, 64, dtype=torch.bfloat16, device="cuda"), pos[:1])
+    assert e.value.status == binding.ERR_ARG
+    assert c.status() == binding.OK
+    before = c.query()
+    c.append(0, K, K, ty, pos + 40)                       # 80 > capacity 64: dropped on the device
+    assert c.status() == binding.ERR_CAPACITY
+    after = c.query()
+    assert np.array_equal(before["gids"], after["gids"])
+    with pytest.raises(binding.SvlmError) as e:
+        c.append(0, torch.zeros(100, 1, 64, dtype=torch.bfloat16, device="cuda"),
+                 torch.zeros(100, 1, 64, dtype=torch.bfloat16, device="cuda"),
+                 torch.zeros(100, dtype=torch.uint8, device="cuda"), torch.arange(100, dtype=torch.int32, device="cuda"))
+    assert e.value.status == binding.ERR_CAPACITY
