@@ -38,13 +38,17 @@ __global__ void __launch_bounds__(256) kv_write_kernel(SvlmCacheDev cd, int laye
     const int i = t / groups, g = t % groups;
     if (i >= n) return;
     const int slot = cd.new_slot[i];
+    // A layer's keys may arrive after an eviction has already shifted these tokens (layers are
+    // computed one after another): rotate at the slot's CURRENT position, and skip a token that
+    // the eviction has dropped in the meantime.
+    if (cd.slot_gid[slot] != cd.ctrl->n_total - n + i) return;
     float cs[8], sn[8];
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
         const int pair = g * 8 + j;
         const int axis = cd.rope_mode == 0 ? 0 : (pair < cd.sec_t ? 0 : (pair < cd.sec_th ? 1 : 2));
         double s, c;
-        sincos((double)cd.new_c[3 * i + axis] * cd.theta[pair], &s, &c);
+        sincos((double)cd.slot_c[axis * cd.n_slots + slot] * cd.theta[pair], &s, &c);
         cs[j] = (float)c;
         sn[j] = (float)s;
     }

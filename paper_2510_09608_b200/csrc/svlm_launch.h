@@ -18,3 +18,9 @@ void svlm_launch_evict_rotate(const SvlmCacheDev& cd, cudaStream_t st);
 // Q, out: [n_caches][n_layers][n_q][q_heads][d]; q_pos: [n_caches][n_q](x3)
 void svlm_launch_attend_simple(const SvlmAttendBatch& b, int layer0, int n_layers, const void* Q, const int* q_pos,
                                int n_q, int q_heads, void* out, cudaStream_t st);
+
+// split-KV decode, n_q = 1 (svlm_decode.cu)
+size_t svlm_decode_ws_floats(int layers_in_launch, int kv_heads, int head_dim, int splits);
+int svlm_decode_splits(int n_pages, int kv_heads, int problems);
+cudaError_t svlm_launch_decode(const SvlmAttendBatch& b, int layer0, int n_layers, const void* Q, const int* q_pos,
+                               int q_heads, void* out, int splits, cudaStream_t st);

@@ -119,6 +119,13 @@ int attend_common(svlm_cache* const* caches, int n_caches, int layer, const void
     DeviceGuard guard(c0->device);
     const int layer0 = layer < 0 ? 0 : layer;
     const int n_layers = layer < 0 ? c0->dev.layers : 1;
+    const int group = q_heads / c0->dev.kv_heads;
+    if (n_q == 1 && group <= 8) {
+        // split-KV decode; every cache's scratch was sized for this launch shape at creation
+        const int splits = svlm_decode_splits(c0->dev.n_pages, c0->dev.kv_heads, n_caches * n_layers);
+        SVLM_CUDA(svlm_launch_decode(b, layer0, n_layers, Q, q_pos, q_heads, out, splits, c0->stream));
+        return SVLM_OK;
+    }
     svlm_launch_attend_simple(b, layer0, n_layers, Q, q_pos, n_q, q_heads, out, c0->stream);
     SVLM_CUDA(cudaGetLastError());
     return SVLM_OK;
@@ -170,6 +177,11 @@ int svlm_cache_create(svlm_cache** out, int layers, int kv_heads, int head_dim, 
     for (int t = 0; t < 2; ++t) {
         A(dev_alloc(c, &d.ev_gid[t], capacity));
         A(dev_alloc(c, &d.ev_pref[t], (size_t)capacity + 1));
+    }
+    {   // split-KV scratch: the larger of a one-layer launch and an all-layers launch
+        const size_t one = svlm_decode_ws_floats(layers, kv_heads, head_dim, svlm_decode_splits(d.n_pages, kv_heads, 1));
+        const size_t all = svlm_decode_ws_floats(layers, kv_heads, head_dim, svlm_decode_splits(d.n_pages, kv_heads, layers));
+        A(dev_alloc(c, &d.ws, std::max(one, all)));
     }
     A(dev_alloc(c, &d.K, slab));
     A(dev_alloc(c, &d.V, slab));

@@ -61,6 +61,18 @@ class SideBySide:
         self.ref.append(None, None, types, pos)
         self.last = (gids, types, pos)
 
+    def append_chunk_first_layer(self):
+        """Layer-sequential use: the chunk's metadata and layer-0 K/V now; other layers after the evict."""
+        gids, types, pos = self.stream.next_chunk()
+        self.cache.append(0, bits_to_dev(self.stream.k(0, gids)), bits_to_dev(self.stream.v(0, gids)),
+                          torch.from_numpy(types).cuda(), torch.from_numpy(np.ascontiguousarray(pos)).cuda())
+        self.ref.append(None, None, types, pos)
+        self.last = (gids, types, pos)
+
+    def append_later_layer(self, layer):
+        gids = self.last[0]
+        self.cache.append(layer, bits_to_dev(self.stream.k(layer, gids)), bits_to_dev(self.stream.v(layer, gids)))
+
     def append_chunk(self, per_layer_calls=False):
         self._append(*self.stream.next_chunk(), per_layer_calls=per_layer_calls)
 

@@ -59,6 +59,27 @@ def test_scaled_mrope_stream_multi_layer(sink_any, contiguous):
     s.check_kv(1)
 
 
+def test_layer_sequential_appends_after_the_evict():
+    """A decoder computes layer l's K/V only after layer l-1 has attended: the chunk's metadata and
+    layer 0 go in first, the eviction runs, and layers 1.. are appended afterwards."""
+    from harness import SideBySide, assert_close
+    wl = dataclasses.replace(_wl(2), layers=3, n_sink=20, vision_window=256, text_window=40,
+                             frames=2, grid_h=8, grid_w=8, text_max=24, decode_steps=2)
+    s = SideBySide(wl)
+    for chunk in range(8):
+        s.append_chunk_first_layer()
+        s.evict()
+        s.check_metadata()
+        assert_close(s.attend(0))
+        for l in (1, 2):
+            s.append_later_layer(l)
+            assert_close(s.attend(l))
+        s.check_kv(chunk % 3)
+        for _ in range(wl.decode_steps):
+            s.append_decode_token()
+            assert_close(s.attend(chunk % 3))
+
+
 @pytest.mark.parametrize("S,Vw,Tw", [(0, 64, 16), (8, 0, 16), (8, 64, 0), (0, 0, 0), (300, 64, 16)])
 def test_degenerate_policies(S, Vw, Tw):
     """Window and sink sizes of zero (the paper's ablation grid has 0-sized sinks and windows), and
