@@ -1,0 +1,453 @@
+#!/usr/bin/env python
+"""Benchmark of the per-chunk KV-cache step (append -> evict -> chunk-prefill -> decode steps).
+
+A "step" is one pass of the whole hot path over one one-second chunk of a synthetic stream in
+steady state: the chunk's tokens are appended, the cache is evicted/re-indexed, every layer attends
+with the chunk's queries, and `decode_steps` single-token decode steps follow (each appends one text
+token and attends in every layer).  Layers are called one after another, as a decoder would.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config 3] [--impl ours|reference]
+
+Prints one JSON line (rank 0).  `--impl reference` times the CPU checker in oracle/ instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2510_09608_b200 import streamgen as sg  # noqa: E402
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return dict(hbm=d["hbm_gbs"], bf16_burst=d["bf16_tflops"], bf16_sustained=d["bf16_tflops_sustained"],
+                    source="measured")
+    return dict(hbm=6650.0, bf16_burst=1590.0, bf16_sustained=1400.0, source="fallback")
+
+
+# ------------------------------------------------------------------------------------------------
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons of one GPU through NVML while the timed region runs."""
+
+    def __init__(self, torch_device_index: int, period=0.05):
+        super().__init__(daemon=True)
+        self.period = period
+        self.samples, self.reasons = [], set()
+        self.max_mhz = None
+        self._halt = threading.Event()
+        self.h = None
+        try:
+            import pynvml
+            import torch
+            pynvml.nvmlInit()
+            uuid = str(torch.cuda.get_device_properties(torch_device_index).uuid)
+            for i in range(pynvml.nvmlDeviceGetCount()):
+                h = pynvml.nvmlDeviceGetHandleByIndex(i)
+                u = pynvml.nvmlDeviceGetUUID(h)
+                u = u.decode() if isinstance(u, bytes) else u
+                if uuid in u:
+                    self.h = h
+            if self.h is None:
+                self.h = pynvml.nvmlDeviceGetHandleByIndex(torch_device_index)
+            self.nv = pynvml
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception as e:  # NVML missing: report that instead of a clock record
+            self.err = repr(e)
+
+    NAMES = {0x1: "gpu_idle", 0x2: "applications_clocks_setting", 0x4: "sw_power_cap", 0x8: "hw_slowdown",
+             0x10: "sync_boost", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown",
+             0x80: "hw_power_brake_slowdown", 0x100: "display_clock_setting"}
+
+    def run(self):
+        if self.h is None:
+            return
+        while not self._halt.is_set():
+            try:
+                self.samples.append(self.nv.nvmlDeviceGetClockInfo(self.h, self.nv.NVML_CLOCK_SM))
+                r = self.nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for bit, name in self.NAMES.items():
+                    if r & bit and name != "gpu_idle":
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def finish(self):
+        self._halt.set()
+        self.join(timeout=2)
+        if self.h is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "note": "NVML unavailable"}
+        return {"sm_mhz": statistics.median(self.samples) if self.samples else None, "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+# ------------------------------------------------------------------------------------------------
+class StepInputs:
+    """Device (and optionally pinned host) inputs of one step, generated from the stream's seed."""
+
+    def __init__(self, wl, stream, chunk, decode, host=False):
+        import torch
+        L = wl.layers
+        gids, types, pos = chunk
+        gen = lambda tensor, g, heads: torch.stack(  # noqa: E731
+            [sg.rows_bf16_torch(wl.seed, tensor, stream.stream, l, g, heads, wl.head_dim) for l in range(L)])
+        self.n = len(gids)
+        self.K, self.V, self.Q = gen(sg.TENSOR_K, gids, wl.kv_heads), gen(sg.TENSOR_V, gids, wl.kv_heads), \
+            gen(sg.TENSOR_Q, gids, wl.q_heads)
+        self.types = torch.from_numpy(types).cuda()
+        self.pos = torch.from_numpy(np.ascontiguousarray(pos)).cuda()
+        self.out = torch.empty_like(self.Q)
+        self.dec = []
+        for g1, t1, p1 in decode:
+            self.dec.append(dict(K=gen(sg.TENSOR_K, g1, wl.kv_heads), V=gen(sg.TENSOR_V, g1, wl.kv_heads),
+                                 Q=gen(sg.TENSOR_Q, g1, wl.q_heads), types=torch.from_numpy(t1).cuda(),
+                                 pos=torch.from_numpy(np.ascontiguousarray(p1)).cuda()))
+            self.dec[-1]["out"] = torch.empty_like(self.dec[-1]["Q"])
+        if host:
+            pin = lambda t: t.cpu().pin_memory()  # noqa: E731
+            self.h = dict(K=pin(self.K), V=pin(self.V), Q=pin(self.Q), types=pin(self.types), pos=pin(self.pos),
+                          out=torch.empty_like(self.Q, device="cpu").pin_memory())
+            self.hdec = [dict(K=pin(d["K"]), V=pin(d["V"]), Q=pin(d["Q"]), types=pin(d["types"]), pos=pin(d["pos"]),
+                              out=torch.empty_like(d["Q"], device="cpu").pin_memory()) for d in self.dec]
+
+    def h2d_bytes(self):
+        tot = 0
+        for d in [self.h] + self.hdec:
+            tot += sum(d[k].numel() * d[k].element_size() for k in ("K", "V", "Q", "types", "pos"))
+        return tot
+
+    def d2h_bytes(self):
+        return sum(d["out"].numel() * d["out"].element_size() for d in [self.h] + self.hdec)
+
+
+def next_step_schedule(stream, wl):
+    chunk = stream.next_chunk()
+    decode = [stream.next_decode_token() for _ in range(wl.decode_steps)]
+    return chunk, decode
+
+
+def run_step(cache, wl, inp, timers=None):
+    """One step through the C ABI, layers in sequence.  timers: dict name -> list of (start,end) events."""
+    import torch
+    L = wl.layers
+
+    def timed(name, fn):
+        if timers is None:
+            return fn()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        fn()
+        b.record()
+        timers.setdefault(name, []).append((a, b))
+
+    timed("append", lambda: cache.append(0, inp.K[0], inp.V[0], inp.types, inp.pos))
+    timed("evict", lambda: cache.evict())
+    timed("prefill", lambda: cache.attend(0, inp.Q[0], inp.pos, inp.out[0]))
+    for l in range(1, L):
+        timed("append", lambda: cache.append(l, inp.K[l], inp.V[l]))
+        timed("prefill", lambda: cache.attend(l, inp.Q[l], inp.pos, inp.out[l]))
+    for d in inp.dec:
+        timed("append1", lambda: cache.append(0, d["K"][0], d["V"][0], d["types"], d["pos"]))
+        timed("decode", lambda: cache.attend(0, d["Q"][0], d["pos"], d["out"][0]))
+        for l in range(1, L):
+            timed("append1", lambda: cache.append(l, d["K"][l], d["V"][l]))
+            timed("decode", lambda: cache.attend(l, d["Q"][l], d["pos"], d["out"][l]))
+
+
+def run_step_host(cache, wl, inp):
+    """The same step through the host-buffer entry points (all layers per call): copies included."""
+    cache.append_host(-1, inp.h["K"], inp.h["V"], inp.h["types"], inp.h["pos"])
+    cache.evict()
+    cache.attend_host(-1, inp.h["Q"], inp.h["pos"], inp.h["out"])
+    for d in inp.hdec:
+        cache.append_host(-1, d["K"], d["V"], d["types"], d["pos"])
+        cache.attend_host(-1, d["Q"], d["pos"], d["out"])
+
+
+def fill_to_steady_state(cache, wl, stream):
+    """Untimed set-up: stream chunks through append+evict (no attention) until the windows are full."""
+    import torch
+    L = wl.layers
+    gen = lambda tensor, g: torch.stack(  # noqa: E731
+        [sg.rows_bf16_torch(wl.seed, tensor, stream.stream, l, g, wl.kv_heads, wl.head_dim) for l in range(L)])
+    n_text = 0
+    chunks = 0
+    while n_text < wl.n_sink + wl.text_window + 64 or chunks * wl.vision_per_chunk < wl.vision_window + 1:
+        gids, types, pos = stream.next_chunk()
+        extra = [stream.next_decode_token() for _ in range(wl.decode_steps)]
+        cache.append(-1, gen(sg.TENSOR_K, gids), gen(sg.TENSOR_V, gids), torch.from_numpy(types).cuda(),
+                     torch.from_numpy(np.ascontiguousarray(pos)).cuda())
+        cache.evict()
+        if extra:
+            g = np.concatenate([e[0] for e in extra])
+            t = np.concatenate([e[1] for e in extra])
+            p = np.concatenate([e[2] for e in extra])
+            cache.append(-1, gen(sg.TENSOR_K, g), gen(sg.TENSOR_V, g), torch.from_numpy(t).cuda(),
+                         torch.from_numpy(np.ascontiguousarray(p)).cuda())
+        n_text += int((types == sg.TEXT).sum()) + len(extra)
+        chunks += 1
+    return chunks
+
+
+def prefill_flops(wl, n_q, lk):
+    pairs = n_q * (lk - n_q) + n_q * (n_q + 1) // 2
+    return 4 * wl.q_heads * wl.head_dim * pairs
+
+
+# ------------------------------------------------------------------------------------------------
+def oracle_sample(wl, rows=48, decode=2):
+    """Times the CPU checker, as it stands, on a bounded sample of one steady-state step: one layer,
+    `rows` query rows of the chunk prefill and `decode` decode steps; the rest is scaled linearly."""
+    import oracle
+    stream = sg.Stream(wl, 0)
+    ref = oracle.Oracle(1, wl.kv_heads, wl.head_dim, wl.n_sink, wl.vision_window, wl.text_window,
+                        rope_mode=wl.rope_mode, rope_base=wl.rope_base, sections=wl.sections)
+    n_text, chunks = 0, 0
+    while n_text < wl.n_sink + wl.text_window + 64 or chunks * wl.vision_per_chunk < wl.vision_window + 1:
+        gids, types, pos = stream.next_chunk()
+        ref.append(None, None, types, pos)
+        ref.evict()
+        for _ in range(wl.decode_steps):
+            g1, t1, p1 = stream.next_decode_token()
+            ref.append(None, None, t1, p1)
+        n_text += int((types == sg.TEXT).sum()) + wl.decode_steps
+        chunks += 1
+    gids, types, pos = stream.next_chunk()
+    ref.append(None, None, types, pos)
+    kept = ref.query()["gids"]
+    ref.set_kv(0, kept, stream.k(0, kept), stream.v(0, kept))
+    Q = stream.q(0, gids)
+    sel = np.linspace(0, len(gids) - 1, rows).astype(np.int64)
+    t0 = time.perf_counter()
+    ref.evict()
+    t_evict = time.perf_counter() - t0
+    t0 = time.perf_counter()
+    ref.attend(0, Q, pos, sel)
+    t_rows = time.perf_counter() - t0
+    t_dec = 0.0
+    for _ in range(decode):
+        g1, t1, p1 = stream.next_decode_token()
+        ref.append(stream.k(0, g1)[None], stream.v(0, g1)[None], t1, p1)
+        t0 = time.perf_counter()
+        ref.attend(0, stream.q(0, g1), p1)
+        t_dec += time.perf_counter() - t0
+    t_dec /= max(decode, 1)
+    # one step = evict (metadata, shared by the layers) + layers x (prefill of all rows + decode steps)
+    est = t_evict + wl.layers * (t_rows * len(gids) / rows + wl.decode_steps * t_dec)
+    return dict(step_seconds=est, measured_seconds=t_evict + t_rows + t_dec * decode, cores=oracle.threads(),
+                sample=f"1 of {wl.layers} layers, {rows} of {len(gids)} prefill rows, {decode} of {wl.decode_steps} "
+                       f"decode steps of one steady-state chunk; scaled linearly to the full step")
+
+
+# ------------------------------------------------------------------------------------------------
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--config", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-graph", action="store_true", help="replay nothing: plain calls in the timed region")
+    args = ap.parse_args()
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    wl = sg.workloads()[args.config]
+    frames_per_step = wl.frames
+    base = dict(metric="sustainable frames/s of the per-chunk evict+attend step (ms_per_step = per-chunk latency)",
+                unit="frames/s", n_gpus=args.gpus, steps=args.steps, warmup=args.warmup, higher_is_better=True,
+                scaling="weak", vs_baseline=None, dtype="bf16", data="synthetic")
+    config = dict(workload=f"config {args.config} ({wl.name}): {wl.layers} layers, {wl.q_heads}/{wl.kv_heads} heads, "
+                           f"d={wl.head_dim}, sinks {wl.n_sink} / vision window {wl.vision_window} / text window "
+                           f"{wl.text_window}, chunk = {wl.frames}x{wl.grid_h}x{wl.grid_w} vision + U(0..{wl.text_max}) "
+                           f"text tokens, {wl.decode_steps} decode steps per chunk, steady state",
+                  layers="sequential calls per layer", l2="working set (KV of all layers) far exceeds L2; no flush",
+                  replicas="one independent stream per GPU, no collective")
+
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        vals = []
+        info = None
+        for i in range(args.warmup + args.steps):
+            info = oracle_sample(wl, rows=16, decode=1)
+            if i >= args.warmup:
+                vals.append(info["step_seconds"])
+        sec = statistics.mean(vals)
+        v = frames_per_step / sec
+        line = dict(base, impl="reference", value=v, ms_per_step=sec * 1e3, config=config,
+                    cpu_baseline=dict(value=v, unit="frames/s", cores=info["cores"], kind="oracle", sample=info["sample"]),
+                    e2e=dict(value=v, unit="frames/s", h2d_bytes_per_step=0, d2h_bytes_per_step=0), n_gpus=1)
+        print(json.dumps(line))
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2510_09608_b200 import binding
+
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    peaks = load_peaks()
+    stream = sg.Stream(wl, rank)
+    cache = binding.Cache(wl.layers, wl.kv_heads, wl.head_dim, wl.n_sink, wl.vision_window, wl.text_window, wl.capacity)
+    cache.set_rope(wl.rope_mode, wl.rope_base, wl.sections)
+    fill_chunks = fill_to_steady_state(cache, wl, stream)
+    cache.evict()
+    assert cache.status() == binding.OK
+
+    total = args.warmup + args.steps
+    want_e2e = not args.no_e2e
+    inputs = [StepInputs(wl, stream, *next_step_schedule(stream, wl)) for _ in range(total)]
+    prime = StepInputs(wl, stream, *next_step_schedule(stream, wl))   # first step of the per-kernel pass
+    # one plain step on a scratch cache first: one-time function attributes are set outside any capture
+    scratch = binding.Cache(wl.layers, wl.kv_heads, wl.head_dim, wl.n_sink, wl.vision_window, wl.text_window, wl.capacity)
+    scratch.set_rope(wl.rope_mode, wl.rope_base, wl.sections)
+    run_step(scratch, wl, inputs[0])
+    torch.cuda.synchronize()
+    scratch.close()
+
+    graphs, launches = [], []
+    if not args.no_graph:
+        # Capturing only records the launches; the cache's device state is untouched until replay.
+        for inp in inputs:
+            g = torch.cuda.CUDAGraph()
+            before = binding.launch_count()
+            with torch.cuda.graph(g):
+                cache.set_stream(torch.cuda.current_stream())
+                run_step(cache, wl, inp)
+            launches.append(binding.launch_count() - before)
+            graphs.append(g)
+        cache.set_stream(torch.cuda.current_stream())
+
+    def do_step(i):
+        if graphs:
+            graphs[i].replay()
+        else:
+            run_step(cache, wl, inputs[i])
+
+    for i in range(args.warmup):
+        do_step(i)
+    sampler = ClockSampler(local)
+    barrier()
+    sampler.start()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    before = binding.launch_count()
+    ev[0].record()
+    for i in range(args.steps):
+        do_step(args.warmup + i)
+        ev[i + 1].record()
+    barrier()
+    clocks = sampler.finish()
+    gpu_launches = sum(launches[args.warmup:]) if graphs else binding.launch_count() - before
+    step_ms = [ev[i].elapsed_time(ev[i + 1]) for i in range(args.steps)]
+    elapsed_ms = ev[0].elapsed_time(ev[-1])
+    assert cache.status() == binding.OK
+    kept = len(cache.query()["gids"])
+
+    # ---- per-kernel durations on the same stream (plain calls, CUDA events around each call) -----
+    timers = {}
+    prof_steps = 3
+    lk_list = []
+    prof_inputs = [prime] + [StepInputs(wl, stream, *next_step_schedule(stream, wl)) for _ in range(prof_steps - 1)]
+    for inp in prof_inputs:
+        run_step(cache, wl, inp, timers)
+        lk_list.append(inp.n)
+    torch.cuda.synchronize()
+    kern = {k: [a.elapsed_time(b) for a, b in v] for k, v in timers.items()}
+    avg = {k: statistics.mean(v) for k, v in kern.items()}
+    tot = {k: sum(v) / prof_steps for k, v in kern.items()}
+    n_q = statistics.mean(lk_list)
+    lk = wl.retained
+    flops = prefill_flops(wl, int(round(n_q)), lk)
+    kv_bytes_layer = lk * 2 * wl.kv_heads * wl.head_dim * 2
+    moved = wl.retained - wl.n_sink
+    evict_bytes = 2 * moved * wl.kv_heads * wl.head_dim * 2 * wl.layers
+    kernels = {
+        "prefill": dict(bound="tensor", avg_ms=avg["prefill"], per_step_ms=tot["prefill"],
+                        achieved=flops / (avg["prefill"] * 1e-3) / 1e12, unit="TFLOP/s", peak=peaks["bf16_burst"]),
+        "decode": dict(bound="hbm (one layer's KV, L2-sized: latency-bound)", avg_ms=avg["decode"],
+                       per_step_ms=tot["decode"], achieved=kv_bytes_layer / (avg["decode"] * 1e-3) / 1e9, unit="GB/s",
+                       peak=peaks["hbm"]),
+        "evict": dict(bound="hbm", avg_ms=avg["evict"], per_step_ms=tot["evict"],
+                      achieved=evict_bytes / (avg["evict"] * 1e-3) / 1e9, unit="GB/s", peak=peaks["hbm"]),
+        "append": dict(avg_ms=avg["append"], per_step_ms=tot["append"] + tot.get("append1", 0.0)),
+    }
+    for k in ("prefill", "decode", "evict"):
+        kernels[k]["frac"] = kernels[k]["achieved"] / kernels[k]["peak"]
+    dominant = max(("prefill", "decode", "evict"), key=lambda k: kernels[k]["per_step_ms"])
+    kd = kernels[dominant]
+    roofline = dict(bound="tensor" if dominant == "prefill" else "hbm", kernel=dominant, achieved=kd["achieved"],
+                    peak=kd["peak"], unit=kd["unit"], frac=kd["frac"], traffic=None,
+                    peak_source=peaks["source"] + (" (burst bf16)" if dominant == "prefill" else " (copy)"))
+
+    # ---- end to end through the host-buffer entry points -----------------------------------------
+    e2e = None
+    if want_e2e:
+        hin = [StepInputs(wl, stream, *next_step_schedule(stream, wl), host=True) for _ in range(3)]
+        e2e_steps = min(args.steps, 5)
+        run_step_host(cache, wl, hin[0])
+        barrier()
+        t0 = time.perf_counter()
+        for i in range(e2e_steps):
+            run_step_host(cache, wl, hin[1 + i % 2])
+        torch.cuda.synchronize()
+        e2e_s = (time.perf_counter() - t0) / e2e_steps
+        if world > 1:
+            t = torch.tensor([e2e_s], device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e_s = float(t.item())
+        e2e = dict(value=world * frames_per_step / e2e_s, unit="frames/s", ms_per_step=e2e_s * 1e3,
+                   h2d_bytes_per_step=hin[1].h2d_bytes(), d2h_bytes_per_step=hin[1].d2h_bytes(),
+                   api="svlm_cache_append_host / svlm_attend_host, all layers per call, pinned host buffers")
+
+    if world > 1:
+        t = torch.tensor([elapsed_ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        elapsed_ms = float(t.item())
+    ms_per_step = elapsed_ms / args.steps
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        info = oracle_sample(wl)
+        cpu = dict(value=frames_per_step / info["step_seconds"], unit="frames/s", cores=info["cores"], kind="oracle",
+                   sample=info["sample"], est_ms_per_step=info["step_seconds"] * 1e3,
+                   measured_seconds=info["measured_seconds"])
+
+    if rank == 0:
+        third = max(1, args.steps // 3)
+        line = dict(base, value=world * frames_per_step / (ms_per_step * 1e-3), ms_per_step=ms_per_step, config=config,
+                    roofline=roofline, cpu_baseline=cpu, e2e=e2e, gpu_launches=int(gpu_launches), clocks=clocks,
+                    kernels=kernels, decode_tok_s=wl.decode_steps / ((tot["decode"] + tot.get("append1", 0)) * 1e-3),
+                    step_ms=dict(min=min(step_ms), median=statistics.median(step_ms), max=max(step_ms),
+                                 first_third=statistics.median(step_ms[:third]),
+                                 last_third=statistics.median(step_ms[-third:])),
+                    state=dict(fill_chunks=fill_chunks, kept_tokens=kept, cuda_graph=bool(graphs)))
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

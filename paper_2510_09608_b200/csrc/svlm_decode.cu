@@ -301,21 +301,49 @@ decode_kernel(SvlmAttendBatch b, int layer0, int n_layers, const uint16_t* __res
     __syncthreads();
     if (!s_last) return;
     __threadfence();
+    // Phase 1: per-split (m, l) into shared memory, then per-head global max, weights and 1/L.
     const float* parts = ws_parts + (size_t)(li * b.kv_heads + hk) * splits * partial_floats<D>();
-    for (int i = threadIdx.x; i < G * D; i += DEC_THREADS) {
+    float* c_m = reinterpret_cast<float*>(smem);          // [splits][8] -> weights exp2(m - M)
+    float* c_l = c_m + splits * 8;                        // [splits][8]
+    float* c_inv = c_l + splits * 8;                      // [8]
+    for (int i = threadIdx.x; i < splits * 16; i += DEC_THREADS) {
+        const int sp = i >> 4, j = i & 15;
+        const float v = __ldcg(parts + (size_t)sp * partial_floats<D>() + 8 * D + j);
+        (j < 8 ? c_m : c_l)[sp * 8 + (j & 7)] = v;
+    }
+    __syncthreads();
+    if (threadIdx.x < 8) {
+        const int h = threadIdx.x;
+        float M = -INFINITY, L = 0.f;
+        for (int sp = 0; sp < splits; ++sp) M = fmaxf(M, c_m[sp * 8 + h]);
+        for (int sp = 0; sp < splits; ++sp) {
+            const float f = M > -INFINITY ? exp2f(c_m[sp * 8 + h] - M) : 0.f;
+            c_m[sp * 8 + h] = f;
+            L += c_l[sp * 8 + h] * f;
+        }
+        c_inv[h] = L > 0.f ? 1.f / L : 0.f;
+    }
+    __syncthreads();
+    // Phase 2: weighted sum of the split outputs; all loads of a thread are independent.
+    constexpr int PER = 8 * D / DEC_THREADS;
+    float acc[PER];
+#pragma unroll
+    for (int e = 0; e < PER; ++e) acc[e] = 0.f;
+    for (int sp = 0; sp < splits; ++sp) {
+        const float* p = parts + (size_t)sp * partial_floats<D>();
+#pragma unroll
+        for (int e = 0; e < PER; ++e) {
+            const int i = e * DEC_THREADS + threadIdx.x;
+            acc[e] += __ldcg(p + i) * c_m[sp * 8 + i / D];
+        }
+    }
+#pragma unroll
+    for (int e = 0; e < PER; ++e) {
+        const int i = e * DEC_THREADS + threadIdx.x;
         const int h = i / D;
-        float M = -INFINITY;
-        for (int sp = 0; sp < splits; ++sp) M = fmaxf(M, __ldcg(parts + (size_t)sp * partial_floats<D>() + 8 * D + h));
-        float acc = 0.f, L = 0.f;
-        if (M > -INFINITY)
-            for (int sp = 0; sp < splits; ++sp) {
-                const float* p = parts + (size_t)sp * partial_floats<D>();
-                const float f = exp2f(__ldcg(p + 8 * D + h) - M);
-                acc += __ldcg(p + i) * f;
-                L += __ldcg(p + 8 * D + 8 + h) * f;
-            }
-        const float res = L > 0.f ? acc / L : 0.f;
-        out[((size_t)prob * q_heads + hk * G + h) * D + (i % D)] = __bfloat16_as_ushort(__float2bfloat16_rn(res));
+        if (h < G)
+            out[((size_t)prob * q_heads + hk * G + h) * D + (i % D)] =
+                __bfloat16_as_ushort(__float2bfloat16_rn(acc[e] * c_inv[h]));
     }
 }
 
@@ -331,9 +359,10 @@ size_t svlm_decode_ws_floats(int layers, int kv_heads, int head_dim, int splits)
 }
 
 int svlm_decode_splits(int n_pages, int kv_heads, int problems) {
-    // about two CTAs' worth of work items per SM; never more splits than pages
+    // about two CTAs' worth of work items per SM, but at most 16 splits: the combine reads every
+    // split's partial once, and beyond 16 that read costs more than the extra parallelism saves
     int splits = (2 * 148 + kv_heads * problems - 1) / (kv_heads * problems);
-    splits = splits < 1 ? 1 : splits;
+    splits = splits < 1 ? 1 : (splits > 16 ? 16 : splits);
     return splits > n_pages ? n_pages : splits;
 }
 

@@ -220,3 +220,43 @@ class Stream:
 
     def q(self, layer: int, gids) -> np.ndarray:
         return rows_bf16(self.wl.seed, TENSOR_Q, self.stream, layer, gids, self.wl.q_heads, self.wl.head_dim)
+
+
+# ---------------------------------------------------------------------------------------------
+# The same generator with torch integer ops, for producing inputs directly in device memory
+# (bit-identical to rows_bf16; torch is only the array library here).
+
+def _t_lsr(x, k):
+    import torch
+    return (x >> k) & ((1 << (64 - k)) - 1)
+
+
+def _t_const(v: int) -> int:
+    return v - (1 << 64) if v >= (1 << 63) else v
+
+
+def _t_mix64(x):
+    z = x + _t_const(0x9E3779B97F4A7C15)
+    z = (z ^ _t_lsr(z, 30)) * _t_const(0xBF58476D1CE4E5B9)
+    z = (z ^ _t_lsr(z, 27)) * _t_const(0x94D049BB133111EB)
+    return z ^ _t_lsr(z, 31)
+
+
+_T_TABLES = {}
+
+
+def rows_bf16_torch(seed: int, tensor: int, stream: int, layer: int, gids, heads: int, head_dim: int, device="cuda"):
+    """bf16 tensor [len(gids), heads, head_dim] on `device`, bit-identical to rows_bf16."""
+    import torch
+    key = str(device)
+    if key not in _T_TABLES:
+        _T_TABLES[key] = torch.from_numpy(normal_table().view(np.int16)).to(device)
+    table = _T_TABLES[key]
+    g = torch.as_tensor(np.asarray(gids, dtype=np.int64), device=device) if not isinstance(gids, torch.Tensor) else gids
+    k0 = int(mix64(np.uint64(seed) ^ (np.uint64(tensor) << np.uint64(56))))
+    with np.errstate(over="ignore"):
+        k1 = int(mix64(np.uint64(k0) + ((np.uint64(stream) << np.uint64(32)) | np.uint64(layer))))
+    keys = _t_mix64(g + _t_const(k1))
+    e = torch.arange(heads * head_dim, dtype=torch.int64, device=device)
+    idx = _t_lsr(_t_mix64(keys[:, None] + e[None, :]), 48)
+    return table[idx].view(torch.bfloat16).reshape(len(g), heads, head_dim)

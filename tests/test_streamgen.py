@@ -37,3 +37,12 @@ def test_chunk_schedule_shapes():
     wl1 = sg.workloads()[1]
     g, t, p = sg.Stream(wl1).next_chunk()
     assert p.ndim == 1 and (t[:32] == sg.VISION).all() and 32 <= len(g) <= 40
+
+
+def test_torch_generator_is_bit_identical():
+    import torch
+    gids = np.array([0, 1, 17, 123456789, 2 ** 40 + 5])
+    for tensor, heads, d in ((sg.TENSOR_K, 4, 128), (sg.TENSOR_Q, 28, 128), (sg.TENSOR_V, 1, 64)):
+        a = sg.rows_bf16(0x5EED0003, tensor, 5, 27, gids, heads, d)
+        b = sg.rows_bf16_torch(0x5EED0003, tensor, 5, 27, gids, heads, d, device="cpu")
+        assert np.array_equal(a, b.view(torch.int16).numpy().view(np.uint16))
