@@ -66,6 +66,7 @@ struct SvlmCacheDev {        // passed by value to kernels
     uint16_t* K;             // [layers][kv_heads][n_slots][head_dim] bf16, rotated at slot_c
     uint16_t* V;             // same shape, as appended
     float* ws;               // split-KV partials
+    void* tmaps;             // TMA descriptors of the K and V slabs (device memory, 2 x 128 bytes)
     double theta[SVLM_MAX_HALF];   // base^(-2i/head_dim)
 };
 
@@ -76,6 +77,7 @@ struct SvlmAttendView {      // what attention needs from one cache
     const SvlmTile* tiles;
     const long long* slot_gid;
     float* ws;
+    const void* tmaps;       // two 128-byte TMA descriptors in device memory: K slab, then V slab
 };
 
 struct SvlmAttendBatch {     // kernel parameter: up to 32 caches share one launch

@@ -24,3 +24,8 @@ size_t svlm_decode_ws_floats(int layers_in_launch, int kv_heads, int head_dim, i
 int svlm_decode_splits(int n_pages, int kv_heads, int problems);
 cudaError_t svlm_launch_decode(const SvlmAttendBatch& b, int layer0, int n_layers, const void* Q, const int* q_pos,
                                int q_heads, void* out, int splits, cudaStream_t st);
+
+// tcgen05/TMEM/TMA chunk prefill, n_q >= 2 (svlm_prefill_sm100.cu)
+bool svlm_prefill_supported(int n_pages, int group);
+cudaError_t svlm_launch_prefill(const SvlmAttendBatch& b, int layer0, int n_layers, const void* Q, const int* q_pos,
+                                int n_q, int q_heads, void* out, cudaStream_t st);

@@ -2,6 +2,7 @@
 // validates arguments, and enqueues the kernels on the cache's stream.  No host synchronisation on
 // the hot path: everything the kernels need to know about the stream's state lives in the device
 // control block.
+#include <cuda.h>
 #include <cuda_runtime.h>
 
 #include <algorithm>
@@ -83,6 +84,36 @@ void fill_view(const svlm_cache* c, SvlmAttendView& v) {
     v.tiles = c->dev.tiles;
     v.slot_gid = c->dev.slot_gid;
     v.ws = c->dev.ws;
+    v.tmaps = c->dev.tmaps;
+}
+
+// TMA descriptors of the K and V slabs: a 2D view [layers*kv_heads*n_slots rows][head_dim] with a
+// 64-element x 128-row box and 128-byte swizzle (one box = half a page of one head at head_dim 128).
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+int make_tensor_maps(svlm_cache* c) {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn ||
+        qres != cudaDriverEntryPointSuccess)
+        return SVLM_ERR_CUDA;
+    EncodeTiledFn encode = reinterpret_cast<EncodeTiledFn>(fn);
+    const SvlmCacheDev& d = c->dev;
+    alignas(64) CUtensorMap maps[2];
+    for (int which = 0; which < 2; ++which) {
+        cuuint64_t dims[2] = {(cuuint64_t)d.head_dim, (cuuint64_t)d.layers * d.kv_heads * d.n_slots};
+        cuuint64_t strides[1] = {(cuuint64_t)d.head_dim * 2};
+        cuuint32_t box[2] = {64, SVLM_PAGE};
+        cuuint32_t estr[2] = {1, 1};
+        if (encode(&maps[which], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, which ? (void*)d.V : (void*)d.K, dims, strides, box,
+                   estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return SVLM_ERR_CUDA;
+    }
+    if (cudaMemcpy(d.tmaps, maps, sizeof maps, cudaMemcpyHostToDevice) != cudaSuccess) return SVLM_ERR_CUDA;
+    return SVLM_OK;
 }
 
 void fill_batch_geometry(const svlm_cache* c, SvlmAttendBatch& b) {
@@ -124,6 +155,10 @@ int attend_common(svlm_cache* const* caches, int n_caches, int layer, const void
         // split-KV decode; every cache's scratch was sized for this launch shape at creation
         const int splits = svlm_decode_splits(c0->dev.n_pages, c0->dev.kv_heads, n_caches * n_layers);
         SVLM_CUDA(svlm_launch_decode(b, layer0, n_layers, Q, q_pos, q_heads, out, splits, c0->stream));
+        return SVLM_OK;
+    }
+    if (n_q >= 2 && svlm_prefill_supported(c0->dev.n_pages, group)) {
+        SVLM_CUDA(svlm_launch_prefill(b, layer0, n_layers, Q, q_pos, n_q, q_heads, out, c0->stream));
         return SVLM_OK;
     }
     svlm_launch_attend_simple(b, layer0, n_layers, Q, q_pos, n_q, q_heads, out, c0->stream);
@@ -185,6 +220,12 @@ int svlm_cache_create(svlm_cache** out, int layers, int kv_heads, int head_dim, 
     }
     A(dev_alloc(c, &d.K, slab));
     A(dev_alloc(c, &d.V, slab));
+    {
+        unsigned char* tm = nullptr;
+        A(dev_alloc(c, &tm, 256));
+        d.tmaps = tm;
+    }
+    if (rc == SVLM_OK) rc = make_tensor_maps(c);
     if (rc == SVLM_OK) {
         // pool pages on the free stack (top of the stack = lowest page number)
         std::vector<int> stack;
