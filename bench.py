@@ -262,12 +262,16 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="replay nothing: plain calls in the timed region")
+    ap.add_argument("--layers", type=int, default=0, help="override the layer count (smaller case for profiling)")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
     wl = sg.workloads()[args.config]
+    if args.layers:
+        import dataclasses
+        wl = dataclasses.replace(wl, layers=args.layers, name=f"{wl.name}, cut to {args.layers} layers")
     frames_per_step = wl.frames
     base = dict(metric="sustainable frames/s of the per-chunk evict+attend step (ms_per_step = per-chunk latency)",
                 unit="frames/s", n_gpus=args.gpus, steps=args.steps, warmup=args.warmup, higher_is_better=True,
