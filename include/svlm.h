@@ -42,7 +42,8 @@ enum svlm_status {
     SVLM_ERR_ORDER = -3,    /* call sequence invalid (e.g. more queries than tokens appended) */
     SVLM_ERR_CUDA = -4,     /* a CUDA runtime or driver call failed */
     SVLM_ERR_TIMEOUT = -5,  /* a bounded device-side wait ran out */
-    SVLM_ERR_NOMEM = -6     /* device or host allocation failed */
+    SVLM_ERR_NOMEM = -6,    /* device or host allocation failed */
+    SVLM_ERR_TOO_LARGE = -7 /* problem exceeds the fixed scratch of svlm_attend_decode_noalloc */
 };
 
 /*
@@ -140,6 +141,35 @@ int svlm_cache_append_host(svlm_cache* c, int layer, const void* K_host, const v
                            const uint8_t* token_type_host, const int32_t* pos_host, int n);
 int svlm_attend_host(svlm_cache* c, int layer, const void* Q_host, const int32_t* q_pos_host, int n_q, int q_heads,
                      void* out_host);
+
+/*
+ * Decode attention (one query token, as svlm_attend with n_q == 1 and layer >= 0) for callers that
+ * cannot allocate device memory when they attend.  (The paper has no counterpart: this is a
+ * deployment convenience of the library.)
+ * Some hosts of this library may not call the CUDA allocator once they are running: a server that has
+ * given every free byte of the GPU to its own memory pool, a real-time loop that cannot afford the
+ * allocator's device-wide lock, code that runs where allocation calls are forbidden.  svlm_attend
+ * keeps its split-KV partial results in scratch memory that svlm_cache_create allocated; this entry
+ * point uses a fixed array of SVLM_NOALLOC_SCRATCH_BYTES that is part of the library image instead,
+ * and calls neither cudaMalloc nor cudaFree nor anything else that allocates.
+ *   Q, q_pos, out   as for svlm_attend with n_q == 1: bf16 [q_heads][head_dim], int32 [1] or [3],
+ *                   bf16 [q_heads][head_dim]; device pointers owned by the caller
+ *   q_heads         a multiple of kv_heads, at most 8 query heads per KV head
+ * Limits and rules
+ *   - the array is resident on every GPU that loads the library, for the life of the process;
+ *   - kv_heads x (number of KV splits, at most 16) x (8*head_dim + 16) floats plus one counter per
+ *     (layer, kv_head) must fit in it, otherwise SVLM_ERR_TOO_LARGE is returned and nothing runs
+ *     (28 layers x 4 KV heads x head_dim 128 needs about 0.27 MB);
+ *   - all calls on one GPU share the array and it keeps the previous call's contents; the call
+ *     clears what has to start at zero, on the cache's stream, before its kernel.  Calls whose
+ *     kernels can overlap on the GPU (different streams, different caches) race on it: order them;
+ *   - the first call on each GPU looks up the array's device address, which can load the library's
+ *     code on that GPU: make that first call before starting any stream capture.
+ * Errors: SVLM_ERR_ARG, SVLM_ERR_ORDER (nothing appended yet), SVLM_ERR_TOO_LARGE, SVLM_ERR_CUDA.
+ * The result equals svlm_attend's for the same state and inputs.
+ */
+#define SVLM_NOALLOC_SCRATCH_BYTES (1u << 20)
+int svlm_attend_decode_noalloc(svlm_cache* c, int layer, const void* Q, const int32_t* q_pos, int q_heads, void* out);
 
 /*
  * Read back the stored tokens in stream order (HOST output buffers, each may be null; sized for

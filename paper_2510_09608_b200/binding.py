@@ -22,7 +22,7 @@ _lib = C.CDLL(LIB_PATH)
 
 TEXT, VISION = 0, 1
 ROPE_1D, ROPE_MROPE = 0, 1
-OK, ERR_ARG, ERR_CAPACITY, ERR_ORDER, ERR_CUDA, ERR_TIMEOUT, ERR_NOMEM = 0, -1, -2, -3, -4, -5, -6
+OK, ERR_ARG, ERR_CAPACITY, ERR_ORDER, ERR_CUDA, ERR_TIMEOUT, ERR_NOMEM, ERR_TOO_LARGE = 0, -1, -2, -3, -4, -5, -6, -7
 
 _vp, _i, _i64p = C.c_void_p, C.c_int, C.POINTER(C.c_int64)
 _lib.svlm_cache_create.argtypes = [C.POINTER(_vp), _i, _i, _i, _i, _i, _i, _i]
@@ -37,6 +37,7 @@ _lib.svlm_attend.argtypes = [_vp, _i, _vp, _vp, _i, _i, _vp]
 _lib.svlm_attend_batched.argtypes = [C.POINTER(_vp), _i, _i, _vp, _vp, _i, _i, _vp]
 _lib.svlm_cache_append_host.argtypes = [_vp, _i, _vp, _vp, _vp, _vp, _i]
 _lib.svlm_attend_host.argtypes = [_vp, _i, _vp, _vp, _i, _i, _vp]
+_lib.svlm_attend_decode_noalloc.argtypes = [_vp, _i, _vp, _vp, _i, _vp]
 _lib.svlm_cache_query.argtypes = [_vp, _i64p, _vp, _vp, _vp, _i64p]
 _lib.svlm_cache_read_kv.argtypes = [_vp, _i, _vp, _vp]
 _lib.svlm_cache_status.argtypes = [_vp]
@@ -131,6 +132,18 @@ class Cache:
         rc = _lib.svlm_attend(self._h, layer, _dev_ptr(Q, torch.bfloat16), _dev_ptr(q_pos, torch.int32), n_q, q_heads,
                               _dev_ptr(out, torch.bfloat16))
         _check(rc, "svlm_attend")
+        return out
+
+    def attend_decode_noalloc(self, layer, Q, q_pos, out=None):
+        """Decode attention (Q: bf16 CUDA [1, q_heads, d]) through the entry point that allocates nothing in
+        the library: its scratch is a fixed array in the library image.  `out` should be passed by callers
+        that must not allocate at all; it is created here only as a convenience when omitted."""
+        if out is None:
+            out = torch.empty_like(Q)
+        assert Q.shape[-3] == 1
+        rc = _lib.svlm_attend_decode_noalloc(self._h, layer, _dev_ptr(Q, torch.bfloat16), _dev_ptr(q_pos, torch.int32),
+                                             Q.shape[-2], _dev_ptr(out, torch.bfloat16))
+        _check(rc, "svlm_attend_decode_noalloc")
         return out
 
     def append_host(self, layer, K, V, token_type=None, pos=None):

@@ -16,23 +16,11 @@
 
 #include "../../include/svlm.h"
 #include "svlm_dev.h"
+#include "svlm_host.h"
 #include "svlm_launch.h"
 
 static std::atomic<long long> g_launches{0};
 void svlm_count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
-
-struct svlm_cache {
-    SvlmCacheDev dev;
-    cudaStream_t stream = nullptr;
-    int device = 0;
-    std::vector<void*> allocs;
-    long long appended = 0;       // tokens accepted by the host checks so far
-    int pending_n = 0;            // n of the latest metadata append (layers 1.. must match)
-    bool configured_locked = false;
-    // staging for the *_host entry points
-    void* stage = nullptr;
-    size_t stage_bytes = 0;
-};
 
 namespace {
 
@@ -465,6 +453,7 @@ const char* svlm_strerror(int status) {
         case SVLM_ERR_CUDA: return "CUDA call failed";
         case SVLM_ERR_TIMEOUT: return "bounded device wait ran out";
         case SVLM_ERR_NOMEM: return "out of memory";
+        case SVLM_ERR_TOO_LARGE: return "problem exceeds the fixed scratch of the no-allocation entry point";
         default: return "unknown status";
     }
 }
