@@ -123,6 +123,25 @@ int svlm_cache_evict(svlm_cache* c);
 int svlm_attend(svlm_cache* c, int layer, const void* Q, const int32_t* q_pos, int n_q, int q_heads, void* out);
 
 /*
+ * One decode step of one layer in a single launch: append ONE token (the token just generated; paper
+ * Section 2.1 keeps past outputs as previous text) and attend with that token's query, i.e.
+ * svlm_cache_append(c, layer, K, V, token_type, pos, 1) followed by
+ * svlm_attend(c, layer, Q, pos, 1, q_heads, out), with identical results (paper Section 3.3: the
+ * per-token latency of this step over the fixed-length cache is the efficiency figure).
+ *   K, V        bf16 [kv_heads][head_dim], un-rotated     Q, out   bf16 [q_heads][head_dim]
+ *   token_type  uint8 [1], pos int32 [1] or [3]: the metadata is taken by the call with layer 0;
+ *               calls for layers 1.. of the same token follow and may pass null token_type (pos is
+ *               still needed: it is the query's position).
+ * At most 8 query heads per KV head.  Consecutive calls for different layers of the same token
+ * overlap on the GPU (the next layer's cache pages are fetched while the previous layer finishes);
+ * K, V, Q and everything else produced by earlier work in the stream are read only after that work
+ * has completed.
+ * Errors: SVLM_ERR_ARG, SVLM_ERR_ORDER (layer > 0 without a preceding one-token append).
+ */
+int svlm_decode_step(svlm_cache* c, int layer, const void* K, const void* V, const uint8_t* token_type,
+                     const int32_t* pos, const void* Q, int q_heads, void* out);
+
+/*
  * The same for n_caches independent streams in one launch (layer >= 0 only).  All caches must
  * share geometry, RoPE settings, device and stream (the first cache's stream is used).
  * Q and out are [n_caches][n_q][q_heads][head_dim]; q_pos is [n_caches][n_q] or [n_caches][n_q][3].
@@ -157,9 +176,9 @@ int svlm_attend_host(svlm_cache* c, int layer, const void* Q_host, const int32_t
  *   q_heads         a multiple of kv_heads, at most 8 query heads per KV head
  * Limits and rules
  *   - the array is resident on every GPU that loads the library, for the life of the process;
- *   - kv_heads x (number of KV splits, at most 16) x (8*head_dim + 16) floats plus one counter per
- *     (layer, kv_head) must fit in it, otherwise SVLM_ERR_TOO_LARGE is returned and nothing runs
- *     (28 layers x 4 KV heads x head_dim 128 needs about 0.27 MB);
+ *   - kv_heads x (number of KV splits: about one CTA per SM over the KV heads) x (8*head_dim + 16)
+ *     floats plus one counter per (layer, kv_head) must fit in it, otherwise SVLM_ERR_TOO_LARGE is
+ *     returned and nothing runs (28 layers x 4 KV heads x head_dim 128 needs about 0.6 MB);
  *   - all calls on one GPU share the array and it keeps the previous call's contents; the call
  *     clears what has to start at zero, on the cache's stream, before its kernel.  Calls whose
  *     kernels can overlap on the GPU (different streams, different caches) race on it: order them;

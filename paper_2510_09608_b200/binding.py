@@ -34,6 +34,7 @@ _lib.svlm_cache_set_stream.argtypes = [_vp, _vp]
 _lib.svlm_cache_append.argtypes = [_vp, _i, _vp, _vp, _vp, _vp, _i]
 _lib.svlm_cache_evict.argtypes = [_vp]
 _lib.svlm_attend.argtypes = [_vp, _i, _vp, _vp, _i, _i, _vp]
+_lib.svlm_decode_step.argtypes = [_vp, _i, _vp, _vp, _vp, _vp, _vp, _i, _vp]
 _lib.svlm_attend_batched.argtypes = [C.POINTER(_vp), _i, _i, _vp, _vp, _i, _i, _vp]
 _lib.svlm_cache_append_host.argtypes = [_vp, _i, _vp, _vp, _vp, _vp, _i]
 _lib.svlm_attend_host.argtypes = [_vp, _i, _vp, _vp, _i, _i, _vp]
@@ -132,6 +133,16 @@ class Cache:
         rc = _lib.svlm_attend(self._h, layer, _dev_ptr(Q, torch.bfloat16), _dev_ptr(q_pos, torch.int32), n_q, q_heads,
                               _dev_ptr(out, torch.bfloat16))
         _check(rc, "svlm_attend")
+        return out
+
+    def decode_step(self, layer, K, V, token_type, pos, Q, out=None):
+        """Append one token (K, V: bf16 CUDA [1, kv_heads, d]) and attend with its query (Q: [1, q_heads, d])."""
+        if out is None:
+            out = torch.empty_like(Q)
+        rc = _lib.svlm_decode_step(self._h, layer, _dev_ptr(K, torch.bfloat16), _dev_ptr(V, torch.bfloat16),
+                                   _dev_ptr(token_type, torch.uint8), _dev_ptr(pos, torch.int32),
+                                   _dev_ptr(Q, torch.bfloat16), Q.shape[-2], _dev_ptr(out, torch.bfloat16))
+        _check(rc, "svlm_decode_step")
         return out
 
     def attend_decode_noalloc(self, layer, Q, q_pos, out=None):

@@ -1,35 +1,45 @@
-// Split-KV decode attention (n_q = 1): one query token per cache/layer attends over the whole
-// retained cache (paper Section 3.3: per-token latency over a fixed-length context is the figure of
-// merit).  The step streams every stored key and value exactly once, so it is bound by HBM
-// bandwidth; the design is about keeping enough bytes in flight:
-//   * grid = (splits, kv_heads, caches*layers); a CTA owns a contiguous run of active pages;
-//   * each of its 4 warps owns the same 32-key quarter of every page and runs its own 3-stage
-//     cp.async ring (16-byte copies into XOR-swizzled shared memory), so no CTA-wide barrier sits
-//     in the streaming loop;
-//   * the G <= 8 query heads that share a kv head ride in the N dimension of m16n8k16 tensor-core
-//     MMAs (S^T = K Q^T, O^T += V^T P^T), so K and V are read once for the whole group;
-//   * per-warp online softmax with warp-shuffle reductions; warps merge through shared memory;
+// Split-KV decode attention (one query token per cache/layer attends over the whole retained cache;
+// paper Section 3.3: per-token latency over a fixed-length context is the figure of merit), optionally
+// fused with the append of that token's own key and value (one "decode step" of a layer).
+//
+// The step reads every stored key and value exactly once, so it is bound by HBM bandwidth; at
+// 19 MB per layer the data time is a few microseconds and everything serial around it counts:
+//   * grid = (splits, kv_heads, caches*layers), about one CTA per SM; a CTA owns a contiguous run of
+//     32-key sub-tiles of the active-page list;
+//   * one producer thread streams the sub-tiles with TMA (2D boxes of 32 keys x 64 dims, 128-byte
+//     swizzle) through a ring of shared-memory stages, each with a full and an empty mbarrier;
+//     the whole first ring-load is in flight before anything else happens;
+//   * four consumer warps take sub-tiles round-robin; the G <= 8 query heads that share a KV head
+//     ride in the N dimension of m16n8k16 MMAs (S^T = K Q^T, O^T += V^T P^T), so K and V are read
+//     once for the whole group; per-warp online softmax with warp-shuffle reductions;
+//   * rotation factors come from a small table (no sincos in the kernel);
+//   * fused append: the warp that owns the sub-tile holding the new token's slot rotates the new key,
+//     patches the row in shared memory and writes key and value to the cache, so the token needs no
+//     launch of its own and is never read from the cache by the step that writes it;
 //   * split partials (o, m, l) go to scratch; the last CTA of a (cache, layer, kv head) to arrive
-//     combines them (arrival counter, no waiting).
+//     combines them (arrival counter, nobody waits);
+//   * with programmatic dependent launch the next layer's kernel starts its loads while this one
+//     finishes: everything that depends on earlier kernels (query, scratch) is read after the
+//     grid-dependency wait, the cache pages are not (the caller's contract, see the launcher).
+// Every mbarrier wait is bounded; on expiry the CTA records SVLM_ERR_TIMEOUT, drains its copies
+// and leaves.
+#include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include "svlm_dev.h"
 #include "svlm_launch.h"
+#include "svlm_ptx.cuh"
+#include "svlm_rope.cuh"
 
 namespace {
 
-constexpr int DEC_WARPS = 4;
-constexpr int DEC_THREADS = DEC_WARPS * 32;
-constexpr int DEC_STAGES = 3;
-constexpr int SUB = 32;            // keys per warp per page
+using namespace svlm_ptx;
 
-__device__ __forceinline__ void cp_async16(void* smem, const void* gmem) {
-    const unsigned s = (unsigned)__cvta_generic_to_shared(smem);
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(s), "l"(gmem));
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N)); }
+constexpr int DEC_CWARPS = 4;                       // consumer warps
+constexpr int DEC_THREADS = (DEC_CWARPS + 1) * 32;  // + one producer warp
+constexpr int DEC_STAGES = 6;
+constexpr int SUB = 32;                             // keys per sub-tile
+constexpr int DEC_MAX_TILES = 512;
 
 __device__ __forceinline__ void ldmatrix_x4(unsigned& r0, unsigned& r1, unsigned& r2, unsigned& r3, const void* p) {
     const unsigned s = (unsigned)__cvta_generic_to_shared(p);
@@ -64,20 +74,35 @@ __device__ __forceinline__ unsigned pack_bf16(float lo, float hi) {
 template <int D>
 __host__ __device__ constexpr int partial_floats() { return 8 * D + 16; }
 
+struct DecShared {
+    unsigned long long full[DEC_STAGES], empty[DEC_STAGES];
+    int abort_flag;
+    int last;
+    unsigned tile_pk[DEC_MAX_TILES];   // page | lo << 16 | hi << 24
+};
+
+// Position of a 16-byte chunk inside a stage: 64-dim panels of [32 keys][128 B], chunks XOR-swizzled
+// by the key's low three bits (the layout the 128-byte-swizzle TMA box writes).
+__device__ __forceinline__ int sw_off(int key, int chunk) {
+    return (chunk >> 3) * (SUB * 128) + key * 128 + (((chunk & 7) ^ (key & 7)) << 4);
+}
+
 template <int D>
 __global__ void __launch_bounds__(DEC_THREADS, 1)
 decode_kernel(SvlmAttendBatch b, int layer0, int n_layers, const uint16_t* __restrict__ Q,
-              const int* __restrict__ q_pos, int q_heads, uint16_t* __restrict__ out, int splits) {
-    constexpr int ROW_BYTES = D * 2;                 // one key row
-    constexpr int CHUNKS = ROW_BYTES / 16;           // 16-byte chunks per row
-    constexpr int STAGE_BYTES = 2 * SUB * ROW_BYTES; // K then V sub-tile
+              const int* __restrict__ q_pos, int q_heads, uint16_t* __restrict__ out, int splits,
+              const uint16_t* __restrict__ Knew, const uint16_t* __restrict__ Vnew, int early_loads) {
+    constexpr int KB = D / 64;                       // 64-dim panels per row
+    constexpr int PANEL_BYTES = SUB * 128;
+    constexpr int STAGE_BYTES = 2 * KB * PANEL_BYTES;   // K panels then V panels
     constexpr int KSTEPS = D / 16;
     constexpr int DBLK = D / 16;
-    extern __shared__ __align__(128) unsigned char smem[];
-    // [warp][stage][K | V]  then  q rows [8][D] bf16
-    unsigned char* my = smem + (size_t)(threadIdx.x >> 5) * DEC_STAGES * STAGE_BYTES;
-    uint16_t* s_q = reinterpret_cast<uint16_t*>(smem + (size_t)DEC_WARPS * DEC_STAGES * STAGE_BYTES);
-    __shared__ int s_last;
+    constexpr int HALF = D / 2;
+    extern __shared__ unsigned char smem_raw[];
+    DecShared& sh = *reinterpret_cast<DecShared*>(smem_raw);
+    unsigned char* ring = reinterpret_cast<unsigned char*>(
+        (reinterpret_cast<uintptr_t>(smem_raw) + sizeof(DecShared) + 1023) & ~(uintptr_t)1023);
+    uint16_t* s_q = reinterpret_cast<uint16_t*>(ring + DEC_STAGES * STAGE_BYTES);   // [8][D] bf16
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int g = lane >> 2, t = lane & 3;
@@ -87,228 +112,301 @@ decode_kernel(SvlmAttendBatch b, int layer0, int n_layers, const uint16_t* __res
     const int layer = layer0 + li;
     const SvlmAttendView& vw = b.view[ci];
     const int G = q_heads / b.kv_heads;
+    volatile int* abort_flag = &sh.abort_flag;
 
-    const int n_tiles = vw.ctrl->n_tiles;
-    const long long shift = vw.ctrl->shift_total;
-    const int tps = (n_tiles + splits - 1) / splits;
-    const int t0 = min(n_tiles, split * tps), t1 = min(n_tiles, t0 + tps);
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < DEC_STAGES; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], 1); }
+        sh.abort_flag = 0;
+        mbar_init_fence();
+    }
+    // The metadata was written by an earlier kernel in the stream.  When the launcher vouches that
+    // the kernel directly before this one did not write it (early_loads), it is read at once;
+    // otherwise after the grid-dependency wait.
+    pdl_launch_dependents();
+    if (!early_loads) pdl_wait();
+    const int n_tiles = min(__ldcg(&vw.ctrl->n_tiles), DEC_MAX_TILES);
+    for (int i = threadIdx.x; i < n_tiles; i += DEC_THREADS) {
+        const int4 tl = __ldcg(reinterpret_cast<const int4*>(vw.tiles + i));   // page, lo, hi, pad
+        sh.tile_pk[i] = (unsigned)tl.x | ((unsigned)tl.y << 16) | ((unsigned)tl.z << 24);
+    }
+    const long long shift = __ldcg(&vw.ctrl->shift_total);
+    // the new token of a fused step: where it lives and whether it is still stored there
+    int new_slot = -1;
+    if (Knew && warp < DEC_CWARPS) {
+        const int s = __ldcg(vw.new_slot);
+        if (__ldcg(&vw.ctrl->append_n) == 1 && __ldcg(vw.slot_gid + s) == __ldcg(&vw.ctrl->n_total) - 1) new_slot = s;
+    }
+    __syncthreads();
 
-    const uint16_t* Kb = vw.K + ((size_t)layer * b.kv_heads + hk) * b.n_slots * D;
-    const uint16_t* Vb = vw.V + ((size_t)layer * b.kv_heads + hk) * b.n_slots * D;
+    const int total_q = 4 * n_tiles;
+    const int q0 = (int)((long long)split * total_q / splits), q1 = (int)((long long)(split + 1) * total_q / splits);
+    const size_t head_row0 = ((size_t)layer * b.kv_heads + hk) * b.n_slots;
+    const size_t part_floats = partial_floats<D>();
+    float* ws_parts = vw.ws + (((size_t)b.layers * b.kv_heads + 3) & ~(size_t)3);   // after the counters (16-byte aligned)
+    float* part = ws_parts + ((size_t)(li * b.kv_heads + hk) * splits + split) * part_floats;
 
-    // ---- sub-tile loader (this warp's 32 keys of tile ti into its stage) ----------------------
-    auto issue = [&](int it) {   // it = index into this warp's sequence of sub-tiles
-        const int ti = t0 + it;
-        if (ti < t1) {
-            const SvlmTile tl = vw.tiles[ti];
-            const int k0 = warp * SUB;
-            if (k0 < tl.hi && k0 + SUB > tl.lo) {
-                unsigned char* st = my + (it % DEC_STAGES) * STAGE_BYTES;
-                const size_t row0 = (size_t)tl.page * SVLM_PAGE + k0;
-                const unsigned char* gk = reinterpret_cast<const unsigned char*>(Kb + row0 * D);
-                const unsigned char* gv = reinterpret_cast<const unsigned char*>(Vb + row0 * D);
+    auto sub_valid = [&](int q, int& page, int& lo, int& hi) {
+        const unsigned pk = sh.tile_pk[q >> 2];
+        page = pk & 0xFFFF; lo = (pk >> 16) & 0xFF; hi = pk >> 24;
+        const int k0 = (q & 3) * SUB;
+        return k0 < hi && k0 + SUB > lo;
+    };
+
+    if (warp == DEC_CWARPS) {
+        // ================= producer =================
+        if (lane == 0) {
+            const unsigned char* maps = reinterpret_cast<const unsigned char*>(vw.tmaps);
+            const void* tmK = maps + 256;
+            const void* tmV = maps + 384;
+            int it = 0;
+            for (int q = q0; q < q1; ++q) {
+                int page, lo, hi;
+                if (!sub_valid(q, page, lo, hi)) continue;
+                const int st = it % DEC_STAGES;
+                if (!mbar_wait(&sh.empty[st], ((it / DEC_STAGES) & 1) ^ 1, abort_flag)) break;
+                unsigned char* dst = ring + st * STAGE_BYTES;
+                const int y = (int)(head_row0 + (size_t)page * SVLM_PAGE + (q & 3) * SUB);
+                mbar_expect_tx(&sh.full[st], STAGE_BYTES);
 #pragma unroll
-                for (int j = 0; j < SUB * CHUNKS / 32; ++j) {
-                    const int idx = j * 32 + lane;
-                    const int r = idx / CHUNKS, c = idx % CHUNKS;
-                    const int dst = r * ROW_BYTES + ((c ^ (r & 7)) << 4);
-                    cp_async16(st + dst, gk + (size_t)idx * 16);
-                    cp_async16(st + SUB * ROW_BYTES + dst, gv + (size_t)idx * 16);
+                for (int kb = 0; kb < KB; ++kb) {
+                    tma_load_2d(dst + kb * PANEL_BYTES, tmK, kb * 64, y, &sh.full[st]);
+                    tma_load_2d(dst + (KB + kb) * PANEL_BYTES, tmV, kb * 64, y, &sh.full[st]);
+                }
+                ++it;
+            }
+        }
+    } else {
+        // ================= consumers =================
+        if (early_loads) pdl_wait();   // from here on: data that earlier kernels in the stream produced
+        const float2* tab = reinterpret_cast<const float2*>(b.rope_tab);
+        // ---- query rows: rotate at q_pos - shift_total, round to bf16, park in shared memory ----
+        {
+            const int pair = threadIdx.x & (HALF - 1);
+            const int axis = b.rope_mode == 0 ? 0 : (pair < b.sec_t ? 0 : (pair < b.sec_th ? 1 : 2));
+            const int* qp = q_pos + (size_t)ci * (b.rope_mode == 0 ? 1 : 3);
+            const long long c = (long long)qp[b.rope_mode == 0 ? 0 : axis] - shift;
+            const float2 cs = svlm_rope_cs(tab, HALF, pair, c, b.theta[pair]);
+            for (int h = threadIdx.x / HALF; h < 8; h += (DEC_CWARPS * 32) / HALF) {
+                float lo = 0.f, hi = 0.f;
+                if (h < G) {
+                    const size_t off = (((size_t)prob) * q_heads + hk * G + h) * D;   // n_q = 1
+                    const float x = __bfloat162float(__ushort_as_bfloat16(Q[off + pair]));
+                    const float y = __bfloat162float(__ushort_as_bfloat16(Q[off + pair + HALF]));
+                    lo = x * cs.x - y * cs.y;
+                    hi = y * cs.x + x * cs.y;
+                }
+                s_q[h * D + pair] = __bfloat16_as_ushort(__float2bfloat16_rn(lo));
+                s_q[h * D + pair + HALF] = __bfloat16_as_ushort(__float2bfloat16_rn(hi));
+            }
+        }
+        asm volatile("bar.sync 1, %0;" ::"n"(DEC_CWARPS * 32));   // consumer warps only
+        unsigned qf[KSTEPS][2];   // B fragments of Q^T: (d = ks*16 + 2t.., head g)
+#pragma unroll
+        for (int ks = 0; ks < KSTEPS; ++ks) {
+            qf[ks][0] = *reinterpret_cast<const unsigned*>(s_q + g * D + ks * 16 + 2 * t);
+            qf[ks][1] = *reinterpret_cast<const unsigned*>(s_q + g * D + ks * 16 + 2 * t + 8);
+        }
+
+        const float scale = 1.4426950408889634f * rsqrtf((float)D);
+        float o[DBLK][4];
+#pragma unroll
+        for (int i = 0; i < DBLK; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
+        float m[2] = {-INFINITY, -INFINITY}, l[2] = {0.f, 0.f};   // heads 2t, 2t+1 (l: this thread's share)
+
+        int it = 0;
+        bool ok = true;
+        for (int q = q0; q < q1 && ok; ++q) {
+            int page, lo, hi;
+            if (!sub_valid(q, page, lo, hi)) continue;
+            const int my = (it % DEC_CWARPS) == warp;
+            const int st = it % DEC_STAGES;
+            const unsigned par = (it / DEC_STAGES) & 1;
+            ++it;
+            if (!my) continue;
+            ok = mbar_wait(&sh.full[st], par, abort_flag);
+            if (!ok) break;
+            unsigned char* sk = ring + st * STAGE_BYTES;
+            unsigned char* sv = sk + KB * PANEL_BYTES;
+            const int k0 = (q & 3) * SUB;
+
+            if (new_slot >= 0 && (new_slot >> 7) == page && ((new_slot & 127) >> 5) == (q & 3)) {
+                // fused append: rotate the new key at its position, put key and value into the
+                // shared-memory row and into the cache
+                const int r = new_slot & 31;
+                const uint16_t* ksrc = Knew + ((size_t)prob * b.kv_heads + hk) * D;
+                const uint16_t* vsrc = Vnew + ((size_t)prob * b.kv_heads + hk) * D;
+                uint16_t* kdst = const_cast<uint16_t*>(vw.K) + (head_row0 + new_slot) * D;
+                uint16_t* vdst = const_cast<uint16_t*>(vw.V) + (head_row0 + new_slot) * D;
+                for (int pair = lane; pair < HALF; pair += 32) {
+                    const int axis = b.rope_mode == 0 ? 0 : (pair < b.sec_t ? 0 : (pair < b.sec_th ? 1 : 2));
+                    const long long c = __ldcg(vw.slot_c + (size_t)axis * b.n_slots + new_slot);
+                    const float2 cs = svlm_rope_cs(tab, HALF, pair, c, b.theta[pair]);
+                    const float x = __bfloat162float(__ushort_as_bfloat16(ksrc[pair]));
+                    const float y = __bfloat162float(__ushort_as_bfloat16(ksrc[pair + HALF]));
+                    const uint16_t klo = __bfloat16_as_ushort(__float2bfloat16_rn(x * cs.x - y * cs.y));
+                    const uint16_t khi = __bfloat16_as_ushort(__float2bfloat16_rn(y * cs.x + x * cs.y));
+                    const uint16_t vlo = vsrc[pair], vhi = vsrc[pair + HALF];
+                    kdst[pair] = klo; kdst[pair + HALF] = khi;
+                    vdst[pair] = vlo; vdst[pair + HALF] = vhi;
+                    const int e0 = pair, e1 = pair + HALF;
+                    *reinterpret_cast<uint16_t*>(sk + sw_off(r, e0 >> 3) + (e0 & 7) * 2) = klo;
+                    *reinterpret_cast<uint16_t*>(sk + sw_off(r, e1 >> 3) + (e1 & 7) * 2) = khi;
+                    *reinterpret_cast<uint16_t*>(sv + sw_off(r, e0 >> 3) + (e0 & 7) * 2) = vlo;
+                    *reinterpret_cast<uint16_t*>(sv + sw_off(r, e1 >> 3) + (e1 & 7) * 2) = vhi;
+                }
+                __syncwarp();
+            }
+
+            // S^T[32 keys x 8 heads] = K Q^T
+            float s[2][4];
+#pragma unroll
+            for (int mb = 0; mb < 2; ++mb) {
+                s[mb][0] = s[mb][1] = s[mb][2] = s[mb][3] = 0.f;
+#pragma unroll
+                for (int ks = 0; ks < KSTEPS; ++ks) {
+                    const int i = lane >> 3, r = lane & 7;
+                    const int key = mb * 16 + (i & 1) * 8 + r;
+                    const int chunk = ks * 2 + (i >> 1);
+                    unsigned a0, a1, a2, a3;
+                    ldmatrix_x4(a0, a1, a2, a3, sk + sw_off(key, chunk));
+                    mma_bf16(s[mb], a0, a1, a2, a3, qf[ks][0], qf[ks][1]);
                 }
             }
-        }
-        cp_async_commit();
-    };
-    for (int s = 0; s < DEC_STAGES - 1; ++s) issue(s);
-
-    // ---- query rows: rotate at q_pos - shift_total, round to bf16, park in shared memory -------
-    {
-        const int half = D / 2;
-        for (int i = threadIdx.x; i < 8 * half; i += DEC_THREADS) {
-            const int h = i / half, pair = i % half;
-            float lo = 0.f, hi = 0.f;
-            if (h < G) {
-                const size_t off = (((size_t)prob) * q_heads + hk * G + h) * D;   // n_q = 1
-                const float x = __bfloat162float(__ushort_as_bfloat16(Q[off + pair]));
-                const float y = __bfloat162float(__ushort_as_bfloat16(Q[off + pair + half]));
-                const int axis = b.rope_mode == 0 ? 0 : (pair < b.sec_t ? 0 : (pair < b.sec_th ? 1 : 2));
-                const int* qp = q_pos + (size_t)ci * (b.rope_mode == 0 ? 1 : 3);
-                const long long c = (long long)qp[b.rope_mode == 0 ? 0 : axis] - shift;
-                double sn, cs;
-                sincos((double)c * b.theta[pair], &sn, &cs);
-                lo = x * (float)cs - y * (float)sn;
-                hi = y * (float)cs + x * (float)sn;
+            // scale, mask slots outside [lo, hi), column (head) maxima over the 32 keys
+            float mx[2] = {-INFINITY, -INFINITY};
+#pragma unroll
+            for (int mb = 0; mb < 2; ++mb)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const int key = k0 + mb * 16 + g + (e >> 1) * 8;
+                    const bool in = key >= lo && key < hi;
+                    s[mb][e] = in ? s[mb][e] * scale : -INFINITY;
+                    mx[e & 1] = fmaxf(mx[e & 1], s[mb][e]);
+                }
+#pragma unroll
+            for (int sft = 4; sft < 32; sft <<= 1) {
+                mx[0] = fmaxf(mx[0], __shfl_xor_sync(0xffffffffu, mx[0], sft));
+                mx[1] = fmaxf(mx[1], __shfl_xor_sync(0xffffffffu, mx[1], sft));
             }
-            s_q[h * D + pair] = __bfloat16_as_ushort(__float2bfloat16_rn(lo));
-            s_q[h * D + pair + half] = __bfloat16_as_ushort(__float2bfloat16_rn(hi));
-        }
-    }
-    __syncthreads();
-    unsigned qf[KSTEPS][2];   // B fragments of Q^T: (d = ks*16 + 2t.., head g)
+            float corr[2], mu[2];
 #pragma unroll
-    for (int ks = 0; ks < KSTEPS; ++ks) {
-        qf[ks][0] = *reinterpret_cast<const unsigned*>(s_q + g * D + ks * 16 + 2 * t);
-        qf[ks][1] = *reinterpret_cast<const unsigned*>(s_q + g * D + ks * 16 + 2 * t + 8);
-    }
-
-    const float scale = 1.4426950408889634f * rsqrtf((float)D);
-    float o[DBLK][4];
-#pragma unroll
-    for (int i = 0; i < DBLK; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
-    float m[2] = {-INFINITY, -INFINITY}, l[2] = {0.f, 0.f};   // heads 2t, 2t+1 (l: this thread's share)
-
-    // ---- streaming loop ----------------------------------------------------------------------
-    const int n_it = t1 - t0;
-    for (int it = 0; it < n_it; ++it) {
-        __syncwarp();   // every lane has finished reading the stage that is refilled next
-        issue(it + DEC_STAGES - 1);
-        cp_async_wait<DEC_STAGES - 1>();
-        __syncwarp();
-        const SvlmTile tl = vw.tiles[t0 + it];
-        const int k0 = warp * SUB;
-        if (!(k0 < tl.hi && k0 + SUB > tl.lo)) continue;
-        const unsigned char* sk = my + (it % DEC_STAGES) * STAGE_BYTES;
-        const unsigned char* sv = sk + SUB * ROW_BYTES;
-
-        // S^T[32 keys x 8 heads] = K Q^T
-        float s[2][4];
-#pragma unroll
-        for (int mb = 0; mb < 2; ++mb) {
-            s[mb][0] = s[mb][1] = s[mb][2] = s[mb][3] = 0.f;
-#pragma unroll
-            for (int ks = 0; ks < KSTEPS; ++ks) {
-                const int i = lane >> 3, r = lane & 7;
-                const int key = mb * 16 + (i & 1) * 8 + r;
-                const int chunk = ks * 2 + (i >> 1);
-                unsigned a0, a1, a2, a3;
-                ldmatrix_x4(a0, a1, a2, a3, sk + key * ROW_BYTES + ((chunk ^ (key & 7)) << 4));
-                mma_bf16(s[mb], a0, a1, a2, a3, qf[ks][0], qf[ks][1]);
+            for (int c = 0; c < 2; ++c) {
+                const float mn = fmaxf(m[c], mx[c]);
+                mu[c] = mn == -INFINITY ? 0.f : mn;
+                corr[c] = exp2f(m[c] - mu[c]);      // m = -inf gives 0
+                m[c] = mn;
+                l[c] *= corr[c];
             }
-        }
-        // scale, mask slots outside [lo, hi), column (head) maxima over the 32 keys
-        float mx[2] = {-INFINITY, -INFINITY};
+            unsigned pb[2][2];   // P^T as B fragments: [key block of 16][k halves]
 #pragma unroll
-        for (int mb = 0; mb < 2; ++mb)
+            for (int mb = 0; mb < 2; ++mb) {
+                float p[4];
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const int key = k0 + mb * 16 + g + (e >> 1) * 8;
-                const bool ok = key >= tl.lo && key < tl.hi;
-                s[mb][e] = ok ? s[mb][e] * scale : -INFINITY;
-                mx[e & 1] = fmaxf(mx[e & 1], s[mb][e]);
+                for (int e = 0; e < 4; ++e) {
+                    p[e] = exp2f(s[mb][e] - mu[e & 1]);
+                    l[e & 1] += p[e];
+                }
+                pb[mb][0] = movmatrix_trans(pack_bf16(p[0], p[1]));
+                pb[mb][1] = movmatrix_trans(pack_bf16(p[2], p[3]));
             }
+            // O^T[D x 8 heads] = O^T * corr + V^T P^T
 #pragma unroll
-        for (int sh = 4; sh < 32; sh <<= 1) {
-            mx[0] = fmaxf(mx[0], __shfl_xor_sync(0xffffffffu, mx[0], sh));
-            mx[1] = fmaxf(mx[1], __shfl_xor_sync(0xffffffffu, mx[1], sh));
-        }
-        float corr[2], mu[2];
+            for (int db = 0; db < DBLK; ++db) {
+                o[db][0] *= corr[0]; o[db][2] *= corr[0];
+                o[db][1] *= corr[1]; o[db][3] *= corr[1];
 #pragma unroll
-        for (int c = 0; c < 2; ++c) {
-            const float mn = fmaxf(m[c], mx[c]);
-            mu[c] = mn == -INFINITY ? 0.f : mn;
-            corr[c] = exp2f(m[c] - mu[c]);      // m = -inf gives 0
-            m[c] = mn;
-            l[c] *= corr[c];
-        }
-        unsigned pb[2][2];   // P^T as B fragments: [key block of 16][k halves]
-#pragma unroll
-        for (int mb = 0; mb < 2; ++mb) {
-            float p[4];
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                p[e] = exp2f(s[mb][e] - mu[e & 1]);
-                l[e & 1] += p[e];
+                for (int kb = 0; kb < 2; ++kb) {
+                    const int i = lane >> 3, r = lane & 7;
+                    const int key = kb * 16 + (i >> 1) * 8 + r;
+                    const int chunk = db * 2 + (i & 1);
+                    unsigned a0, a1, a2, a3;
+                    ldmatrix_x4_trans(a0, a1, a2, a3, sv + sw_off(key, chunk));
+                    mma_bf16(o[db], a0, a1, a2, a3, pb[kb][0], pb[kb][1]);
+                }
             }
-            pb[mb][0] = movmatrix_trans(pack_bf16(p[0], p[1]));
-            pb[mb][1] = movmatrix_trans(pack_bf16(p[2], p[3]));
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sh.empty[st]);
         }
-        // O^T[D x 8 heads] = O^T * corr + V^T P^T
+        // l: sum the shares of the 8 lane groups that hold the same heads
+#pragma unroll
+        for (int sft = 4; sft < 32; sft <<= 1) {
+            l[0] += __shfl_xor_sync(0xffffffffu, l[0], sft);
+            l[1] += __shfl_xor_sync(0xffffffffu, l[1], sft);
+        }
+        // ---- merge the consumer warps: s_o[warp][8 heads][D], s_m/s_l[warp][8] (own region, after s_q)
+        float* s_o = reinterpret_cast<float*>(s_q + 8 * D);
+        float* s_m = s_o + DEC_CWARPS * 8 * D;
+        float* s_l = s_m + DEC_CWARPS * 8;
 #pragma unroll
         for (int db = 0; db < DBLK; ++db) {
-            o[db][0] *= corr[0]; o[db][2] *= corr[0];
-            o[db][1] *= corr[1]; o[db][3] *= corr[1];
-#pragma unroll
-            for (int kb = 0; kb < 2; ++kb) {
-                const int i = lane >> 3, r = lane & 7;
-                const int key = kb * 16 + (i >> 1) * 8 + r;
-                const int chunk = db * 2 + (i & 1);
-                unsigned a0, a1, a2, a3;
-                ldmatrix_x4_trans(a0, a1, a2, a3, sv + key * ROW_BYTES + ((chunk ^ (key & 7)) << 4));
-                mma_bf16(o[db], a0, a1, a2, a3, pb[kb][0], pb[kb][1]);
-            }
+            float* base = s_o + (size_t)warp * 8 * D;
+            base[(2 * t) * D + db * 16 + g] = o[db][0];
+            base[(2 * t + 1) * D + db * 16 + g] = o[db][1];
+            base[(2 * t) * D + db * 16 + g + 8] = o[db][2];
+            base[(2 * t + 1) * D + db * 16 + g + 8] = o[db][3];
         }
-    }
-    cp_async_wait<0>();
-    // l: sum the shares of the 8 lane groups that hold the same heads
+        if (g == 0) {
+            s_m[warp * 8 + 2 * t] = m[0]; s_m[warp * 8 + 2 * t + 1] = m[1];
+            s_l[warp * 8 + 2 * t] = l[0]; s_l[warp * 8 + 2 * t + 1] = l[1];
+        }
+        asm volatile("bar.sync 1, %0;" ::"n"(DEC_CWARPS * 32));
+        const int ct = threadIdx.x;   // 0 .. DEC_CWARPS*32-1
+        for (int i = ct; i < 8 * D; i += DEC_CWARPS * 32) {
+            const int h = i / D;
+            float M = -INFINITY;
 #pragma unroll
-    for (int sh = 4; sh < 32; sh <<= 1) {
-        l[0] += __shfl_xor_sync(0xffffffffu, l[0], sh);
-        l[1] += __shfl_xor_sync(0xffffffffu, l[1], sh);
-    }
-    __syncthreads();   // everyone is done with the staging memory: reuse it for the warp merge
-
-    // ---- merge the 4 warps: s_o[warp][8 heads][D], s_m/s_l[warp][8] -----------------------------
-    float* s_o = reinterpret_cast<float*>(smem);
-    float* s_m = s_o + DEC_WARPS * 8 * D;
-    float* s_l = s_m + DEC_WARPS * 8;
+            for (int w = 0; w < DEC_CWARPS; ++w) M = fmaxf(M, s_m[w * 8 + h]);
+            float acc = 0.f;
+            if (M > -INFINITY)
 #pragma unroll
-    for (int db = 0; db < DBLK; ++db) {
-        float* base = s_o + (size_t)warp * 8 * D;
-        base[(2 * t) * D + db * 16 + g] = o[db][0];
-        base[(2 * t + 1) * D + db * 16 + g] = o[db][1];
-        base[(2 * t) * D + db * 16 + g + 8] = o[db][2];
-        base[(2 * t + 1) * D + db * 16 + g + 8] = o[db][3];
-    }
-    if (g == 0) {
-        s_m[warp * 8 + 2 * t] = m[0]; s_m[warp * 8 + 2 * t + 1] = m[1];
-        s_l[warp * 8 + 2 * t] = l[0]; s_l[warp * 8 + 2 * t + 1] = l[1];
-    }
-    __syncthreads();
-    float* ws_parts = vw.ws + (size_t)b.layers * b.kv_heads;   // after the counters
-    float* part = ws_parts + ((size_t)(li * b.kv_heads + hk) * splits + split) * partial_floats<D>();
-    for (int i = threadIdx.x; i < 8 * D; i += DEC_THREADS) {
-        const int h = i / D;
-        float M = -INFINITY;
+                for (int w = 0; w < DEC_CWARPS; ++w) acc += s_o[(size_t)w * 8 * D + i] * exp2f(s_m[w * 8 + h] - M);
+            part[i] = acc;
+        }
+        if (ct < 8) {
+            const int h = ct;
+            float M = -INFINITY, L = 0.f;
 #pragma unroll
-        for (int w = 0; w < DEC_WARPS; ++w) M = fmaxf(M, s_m[w * 8 + h]);
-        float acc = 0.f;
-        if (M > -INFINITY)
+            for (int w = 0; w < DEC_CWARPS; ++w) M = fmaxf(M, s_m[w * 8 + h]);
+            if (M > -INFINITY)
 #pragma unroll
-            for (int w = 0; w < DEC_WARPS; ++w) acc += s_o[(size_t)w * 8 * D + i] * exp2f(s_m[w * 8 + h] - M);
-        part[i] = acc;
-    }
-    if (threadIdx.x < 8) {
-        const int h = threadIdx.x;
-        float M = -INFINITY, L = 0.f;
-#pragma unroll
-        for (int w = 0; w < DEC_WARPS; ++w) M = fmaxf(M, s_m[w * 8 + h]);
-        if (M > -INFINITY)
-#pragma unroll
-            for (int w = 0; w < DEC_WARPS; ++w) L += s_l[w * 8 + h] * exp2f(s_m[w * 8 + h] - M);
-        part[8 * D + h] = M;
-        part[8 * D + 8 + h] = L;
+                for (int w = 0; w < DEC_CWARPS; ++w) L += s_l[w * 8 + h] * exp2f(s_m[w * 8 + h] - M);
+            part[8 * D + h] = M;
+            part[8 * D + 8 + h] = L;
+        }
+        __threadfence();
     }
 
     // ---- last CTA of this (cache, layer, kv head) combines the splits -----------------------------
-    __threadfence();
     __syncthreads();
+    if (sh.abort_flag) {
+        // Somebody gave up.  Copies already issued still land in this CTA's shared memory: give every
+        // full barrier a bounded chance to complete before the memory is released.
+        if (threadIdx.x == 0) {
+            for (int s = 0; s < DEC_STAGES; ++s)
+                for (unsigned p = 0; p < 2; ++p)
+                    for (unsigned w = 0; w < (1u << 16) && !mbar_test(&sh.full[s], p); ++w) __nanosleep(32);
+            atomicCAS(const_cast<int*>(&vw.ctrl->status), 0, -5);   // SVLM_ERR_TIMEOUT
+        }
+        __syncthreads();
+        return;
+    }
     unsigned* counter = reinterpret_cast<unsigned*>(vw.ws) + li * b.kv_heads + hk;
     if (threadIdx.x == 0) {
         const unsigned prev = atomicAdd(counter, 1u);
-        s_last = (prev == (unsigned)splits - 1);
-        if (s_last) *counter = 0;   // ready for the next launch
+        sh.last = (prev == (unsigned)splits - 1);
+        if (sh.last) *counter = 0;   // ready for the next launch
     }
     __syncthreads();
-    if (!s_last) return;
+    if (!sh.last) return;
     __threadfence();
     // Phase 1: per-split (m, l) into shared memory, then per-head global max, weights and 1/L.
-    const float* parts = ws_parts + (size_t)(li * b.kv_heads + hk) * splits * partial_floats<D>();
-    float* c_m = reinterpret_cast<float*>(smem);          // [splits][8] -> weights exp2(m - M)
+    const float* parts = ws_parts + (size_t)(li * b.kv_heads + hk) * splits * part_floats;
+    float* c_m = reinterpret_cast<float*>(ring);          // [splits][8] -> weights exp2(m - M)
     float* c_l = c_m + splits * 8;                        // [splits][8]
     float* c_inv = c_l + splits * 8;                      // [8]
     for (int i = threadIdx.x; i < splits * 16; i += DEC_THREADS) {
         const int sp = i >> 4, j = i & 15;
-        const float v = __ldcg(parts + (size_t)sp * partial_floats<D>() + 8 * D + j);
+        const float v = __ldcg(parts + (size_t)sp * part_floats + 8 * D + j);
         (j < 8 ? c_m : c_l)[sp * 8 + (j & 7)] = v;
     }
     __syncthreads();
@@ -325,50 +423,62 @@ decode_kernel(SvlmAttendBatch b, int layer0, int n_layers, const uint16_t* __res
     }
     __syncthreads();
     // Phase 2: weighted sum of the split outputs; all loads of a thread are independent.
-    constexpr int PER = 8 * D / DEC_THREADS;
-    float acc[PER];
-#pragma unroll
-    for (int e = 0; e < PER; ++e) acc[e] = 0.f;
-    for (int sp = 0; sp < splits; ++sp) {
-        const float* p = parts + (size_t)sp * partial_floats<D>();
-#pragma unroll
-        for (int e = 0; e < PER; ++e) {
-            const int i = e * DEC_THREADS + threadIdx.x;
-            acc[e] += __ldcg(p + i) * c_m[sp * 8 + i / D];
-        }
-    }
-#pragma unroll
-    for (int e = 0; e < PER; ++e) {
-        const int i = e * DEC_THREADS + threadIdx.x;
+    for (int i0 = 0; i0 < 8 * D; i0 += DEC_THREADS * 4) {
+        const int i = i0 + threadIdx.x * 4;
+        if (i >= G * D) continue;
         const int h = i / D;
-        if (h < G)
-            out[((size_t)prob * q_heads + hk * G + h) * D + (i % D)] =
-                __bfloat16_as_ushort(__float2bfloat16_rn(acc[e] * c_inv[h]));
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int sp = 0; sp < splits; ++sp) {
+            const float4 v = __ldcg(reinterpret_cast<const float4*>(parts + (size_t)sp * part_floats + i));
+            const float w = c_m[sp * 8 + h];
+            acc.x += v.x * w; acc.y += v.y * w; acc.z += v.z * w; acc.w += v.w * w;
+        }
+        const float inv = c_inv[h];
+        uint2 pk;
+        pk.x = pack_bf16(acc.x * inv, acc.y * inv);
+        pk.y = pack_bf16(acc.z * inv, acc.w * inv);
+        *reinterpret_cast<uint2*>(out + ((size_t)prob * q_heads + hk * G + h) * D + (i % D)) = pk;
     }
 }
 
 template <int D>
-constexpr size_t decode_smem() { return (size_t)DEC_WARPS * DEC_STAGES * 2 * SUB * D * 2 + 8 * D * 2; }
+constexpr size_t decode_smem() {
+    return sizeof(DecShared) + 1024 + (size_t)DEC_STAGES * 2 * SUB * D * 2 + 8 * D * 2 +
+           (size_t)DEC_CWARPS * 8 * D * 4 + DEC_CWARPS * 16 * 4;
+}
 
 }  // namespace
 
 // Scratch floats needed per cache for `splits` splits (all layers at once is the largest launch).
 size_t svlm_decode_ws_floats(int layers, int kv_heads, int head_dim, int splits) {
     const size_t pf = head_dim == 128 ? partial_floats<128>() : partial_floats<64>();
-    return (size_t)layers * kv_heads + (size_t)layers * kv_heads * splits * pf;
+    return (((size_t)layers * kv_heads + 3) & ~(size_t)3) + (size_t)layers * kv_heads * splits * pf;
 }
 
 int svlm_decode_splits(int n_pages, int kv_heads, int problems) {
-    // about two CTAs' worth of work items per SM, but at most 16 splits: the combine reads every
-    // split's partial once, and beyond 16 that read costs more than the extra parallelism saves
-    int splits = (2 * 148 + kv_heads * problems - 1) / (kv_heads * problems);
-    splits = splits < 1 ? 1 : (splits > 16 ? 16 : splits);
-    return splits > n_pages ? n_pages : splits;
+    // one CTA per SM: the combine reads every split's partial once, so more splits than needed to
+    // fill the machine only lengthen the tail
+    int splits = 148 / (kv_heads * problems);
+    splits = splits < 1 ? 1 : splits;
+    return splits > 4 * n_pages ? 4 * n_pages : splits;
 }
 
 cudaError_t svlm_launch_decode(const SvlmAttendBatch& b, int layer0, int n_layers, const void* Q, const int* q_pos,
-                               int q_heads, void* out, int splits, cudaStream_t st) {
-    dim3 grid(splits, b.kv_heads, b.n_caches * n_layers);
+                               int q_heads, void* out, int splits, const void* Knew, const void* Vnew, int early_loads,
+                               cudaStream_t st) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(splits, b.kv_heads, b.n_caches * n_layers);
+    cfg.blockDim = dim3(DEC_THREADS);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const uint16_t* Qp = (const uint16_t*)Q;
+    uint16_t* Op = (uint16_t*)out;
+    const uint16_t* Kn = (const uint16_t*)Knew;
+    const uint16_t* Vn = (const uint16_t*)Vnew;
     cudaError_t e;
     if (b.head_dim == 128) {
         static bool once = false;
@@ -377,8 +487,9 @@ cudaError_t svlm_launch_decode(const SvlmAttendBatch& b, int layer0, int n_layer
             if (e != cudaSuccess) return e;
             once = true;
         }
-        decode_kernel<128><<<grid, DEC_THREADS, decode_smem<128>(), st>>>(b, layer0, n_layers, (const uint16_t*)Q, q_pos,
-                                                                       q_heads, (uint16_t*)out, splits);
+        cfg.dynamicSmemBytes = decode_smem<128>();
+        e = cudaLaunchKernelEx(&cfg, decode_kernel<128>, b, layer0, n_layers, Qp, q_pos, q_heads, Op, splits, Kn, Vn,
+                               early_loads);
     } else {
         static bool once = false;
         if (!once) {
@@ -386,9 +497,10 @@ cudaError_t svlm_launch_decode(const SvlmAttendBatch& b, int layer0, int n_layer
             if (e != cudaSuccess) return e;
             once = true;
         }
-        decode_kernel<64><<<grid, DEC_THREADS, decode_smem<64>(), st>>>(b, layer0, n_layers, (const uint16_t*)Q, q_pos,
-                                                                     q_heads, (uint16_t*)out, splits);
+        cfg.dynamicSmemBytes = decode_smem<64>();
+        e = cudaLaunchKernelEx(&cfg, decode_kernel<64>, b, layer0, n_layers, Qp, q_pos, q_heads, Op, splits, Kn, Vn,
+                               early_loads);
     }
     svlm_count_launch();
-    return cudaGetLastError();
+    return e != cudaSuccess ? e : cudaGetLastError();
 }

@@ -66,7 +66,9 @@ struct SvlmCacheDev {        // passed by value to kernels
     uint16_t* K;             // [layers][kv_heads][n_slots][head_dim] bf16, rotated at slot_c
     uint16_t* V;             // same shape, as appended
     float* ws;               // split-KV partials
-    void* tmaps;             // TMA descriptors of the K and V slabs (device memory, 2 x 128 bytes)
+    void* tmaps;             // TMA descriptors (device memory, 4 x 128 bytes): K, V slabs with a 128-row box
+                             // (chunk prefill), then K, V with a 32-row box (decode)
+    float* rope_tab;         // [3][256][head_dim/2] (cos, sin) pairs, see svlm_rope.cuh
     double theta[SVLM_MAX_HALF];   // base^(-2i/head_dim)
 };
 
@@ -77,7 +79,9 @@ struct SvlmAttendView {      // what attention needs from one cache
     const SvlmTile* tiles;
     const long long* slot_gid;
     float* ws;
-    const void* tmaps;       // two 128-byte TMA descriptors in device memory: K slab, then V slab
+    const void* tmaps;       // four 128-byte TMA descriptors in device memory (see SvlmCacheDev)
+    const int* new_slot;     // slots of the latest append
+    const int* slot_c;       // [3][n_slots] current positions
 };
 
 struct SvlmAttendBatch {     // kernel parameter: up to 32 caches share one launch
@@ -85,5 +89,6 @@ struct SvlmAttendBatch {     // kernel parameter: up to 32 caches share one laun
     int layers, kv_heads, head_dim, n_slots;
     int rope_mode, sec_t, sec_th;
     SvlmAttendView view[SVLM_MAX_BATCH];
+    const float* rope_tab;   // rotation table of the first cache (all caches of a batch share the geometry)
     double theta[SVLM_MAX_HALF];
 };

@@ -14,6 +14,10 @@ struct svlm_cache {
     long long appended = 0;       // tokens accepted by the host checks so far
     int pending_n = 0;            // n of the latest metadata append (layers 1.. must match)
     bool configured_locked = false;
+    // What the latest enqueued operation was, for the decode step's early loads: a decode of one layer
+    // may start reading its pages while the previous kernel still runs only if that kernel was a decode
+    // of another layer of this cache (which writes neither the metadata nor this layer's pages).
+    int last_decode_layer = -1;   // layer of the latest operation if it was a single-layer decode, else -1
     // staging for the *_host entry points
     void* stage = nullptr;
     size_t stage_bytes = 0;

@@ -22,8 +22,13 @@ void svlm_launch_attend_simple(const SvlmAttendBatch& b, int layer0, int n_layer
 // split-KV decode, n_q = 1 (svlm_decode.cu)
 size_t svlm_decode_ws_floats(int layers_in_launch, int kv_heads, int head_dim, int splits);
 int svlm_decode_splits(int n_pages, int kv_heads, int problems);
+// Knew/Vnew non-null: fused decode step, the latest appended token's key and value ([caches*layers][kv_heads][d],
+// un-rotated) are written to the cache by this launch.  early_loads != 0: the caller vouches that no kernel
+// enqueued since the one before the previous launch on this stream wrote this cache's metadata or the pages of the
+// layers attended here, so the kernel may read them before the previous kernel has finished.
 cudaError_t svlm_launch_decode(const SvlmAttendBatch& b, int layer0, int n_layers, const void* Q, const int* q_pos,
-                               int q_heads, void* out, int splits, cudaStream_t st);
+                               int q_heads, void* out, int splits, const void* Knew, const void* Vnew, int early_loads,
+                               cudaStream_t st);
 
 // tcgen05/TMEM/TMA chunk prefill, n_q >= 2 (svlm_prefill_sm100.cu)
 bool svlm_prefill_supported(int n_pages, int group);

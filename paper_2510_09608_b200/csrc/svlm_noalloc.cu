@@ -63,8 +63,9 @@ extern "C" int svlm_attend_decode_noalloc(svlm_cache* c, int layer, const void* 
 
     const int splits = svlm_decode_splits(d.n_pages, d.kv_heads, 1);
     // counters for every (layer, kv head) of the cache, then one layer's partials
-    const size_t need = ((size_t)(d.layers - 1) * d.kv_heads + svlm_decode_ws_floats(1, d.kv_heads, d.head_dim, splits)) *
-                        sizeof(float);
+    auto up4 = [](size_t x) { return (x + 3) & ~(size_t)3; };
+    const size_t need = (up4((size_t)d.layers * d.kv_heads) - up4((size_t)d.kv_heads) +
+                         svlm_decode_ws_floats(1, d.kv_heads, d.head_dim, splits)) * sizeof(float);
     if (need > kScratchBytes) return SVLM_ERR_TOO_LARGE;
 
     int prev = -1;
@@ -85,9 +86,10 @@ extern "C" int svlm_attend_decode_noalloc(svlm_cache* c, int layer, const void* 
         b.rope_mode = d.rope_mode; b.sec_t = d.sec_t; b.sec_th = d.sec_th;
         std::memcpy(b.theta, d.theta, sizeof b.theta);
         SvlmAttendView& v = b.view[0];
-        v.K = d.K; v.V = d.V; v.ctrl = d.ctrl; v.tiles = d.tiles; v.slot_gid = d.slot_gid; v.tmaps = d.tmaps;
+        v.K = d.K; v.V = d.V; v.ctrl = d.ctrl; v.tiles = d.tiles; v.slot_gid = d.slot_gid; v.tmaps = d.tmaps; v.new_slot = d.new_slot; v.slot_c = d.slot_c;
+        b.rope_tab = d.rope_tab;
         v.ws = scratch;
-        if (svlm_launch_decode(b, layer, 1, Q, q_pos, q_heads, out, splits, c->stream) != cudaSuccess)
+        if (svlm_launch_decode(b, layer, 1, Q, q_pos, q_heads, out, splits, nullptr, nullptr, 0, c->stream) != cudaSuccess)
             rc = SVLM_ERR_CUDA;
     }
     if (prev != c->device) cudaSetDevice(prev);

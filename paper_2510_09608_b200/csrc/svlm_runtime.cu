@@ -73,6 +73,25 @@ void fill_view(const svlm_cache* c, SvlmAttendView& v) {
     v.slot_gid = c->dev.slot_gid;
     v.ws = c->dev.ws;
     v.tmaps = c->dev.tmaps;
+    v.new_slot = c->dev.new_slot;
+    v.slot_c = c->dev.slot_c;
+}
+
+// Rotation table: (cos, sin)(k * 256^level * theta_i) in fp32 from fp64 (see svlm_rope.cuh).
+int upload_rope_table(svlm_cache* c) {
+    const SvlmCacheDev& d = c->dev;
+    const int half = d.head_dim / 2;
+    std::vector<float> tab((size_t)3 * 256 * half * 2);
+    for (int level = 0; level < 3; ++level)
+        for (int k = 0; k < 256; ++k)
+            for (int i = 0; i < half; ++i) {
+                const double ang = (double)k * std::pow(256.0, level) * d.theta[i];
+                tab[(((size_t)level * 256 + k) * half + i) * 2] = (float)std::cos(ang);
+                tab[(((size_t)level * 256 + k) * half + i) * 2 + 1] = (float)std::sin(ang);
+            }
+    if (cudaMemcpy(d.rope_tab, tab.data(), tab.size() * sizeof(float), cudaMemcpyHostToDevice) != cudaSuccess)
+        return SVLM_ERR_CUDA;
+    return SVLM_OK;
 }
 
 // TMA descriptors of the K and V slabs: a 2D view [layers*kv_heads*n_slots rows][head_dim] with a
@@ -89,13 +108,13 @@ int make_tensor_maps(svlm_cache* c) {
         return SVLM_ERR_CUDA;
     EncodeTiledFn encode = reinterpret_cast<EncodeTiledFn>(fn);
     const SvlmCacheDev& d = c->dev;
-    alignas(64) CUtensorMap maps[2];
-    for (int which = 0; which < 2; ++which) {
+    alignas(64) CUtensorMap maps[4];
+    for (int which = 0; which < 4; ++which) {   // K, V with a whole-page box; K, V with a 32-row box
         cuuint64_t dims[2] = {(cuuint64_t)d.head_dim, (cuuint64_t)d.layers * d.kv_heads * d.n_slots};
         cuuint64_t strides[1] = {(cuuint64_t)d.head_dim * 2};
-        cuuint32_t box[2] = {64, SVLM_PAGE};
+        cuuint32_t box[2] = {64, which < 2 ? (cuuint32_t)SVLM_PAGE : 32u};
         cuuint32_t estr[2] = {1, 1};
-        if (encode(&maps[which], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, which ? (void*)d.V : (void*)d.K, dims, strides, box,
+        if (encode(&maps[which], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (which & 1) ? (void*)d.V : (void*)d.K, dims, strides, box,
                    estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return SVLM_ERR_CUDA;
@@ -113,10 +132,11 @@ void fill_batch_geometry(const svlm_cache* c, SvlmAttendBatch& b) {
     b.sec_t = c->dev.sec_t;
     b.sec_th = c->dev.sec_th;
     std::memcpy(b.theta, c->dev.theta, sizeof b.theta);
+    b.rope_tab = c->dev.rope_tab;
 }
 
 int attend_common(svlm_cache* const* caches, int n_caches, int layer, const void* Q, const int32_t* q_pos, int n_q,
-                  int q_heads, void* out) {
+                  int q_heads, void* out, const void* Knew = nullptr, const void* Vnew = nullptr) {
     svlm_cache* c0 = caches[0];
     if (!Q || !q_pos || !out || n_q < 1 || q_heads < 1) return SVLM_ERR_ARG;
     if (q_heads % c0->dev.kv_heads) return SVLM_ERR_ARG;
@@ -139,12 +159,20 @@ int attend_common(svlm_cache* const* caches, int n_caches, int layer, const void
     const int layer0 = layer < 0 ? 0 : layer;
     const int n_layers = layer < 0 ? c0->dev.layers : 1;
     const int group = q_heads / c0->dev.kv_heads;
+    int early = 0;
+    if (n_caches == 1 && n_q == 1 && layer >= 0) {
+        early = c0->last_decode_layer >= 0 && c0->last_decode_layer != layer;
+        c0->last_decode_layer = layer;
+    } else {
+        for (int i = 0; i < n_caches; ++i) caches[i]->last_decode_layer = -1;
+    }
     if (n_q == 1 && group <= 8) {
         // split-KV decode; every cache's scratch was sized for this launch shape at creation
         const int splits = svlm_decode_splits(c0->dev.n_pages, c0->dev.kv_heads, n_caches * n_layers);
-        SVLM_CUDA(svlm_launch_decode(b, layer0, n_layers, Q, q_pos, q_heads, out, splits, c0->stream));
+        SVLM_CUDA(svlm_launch_decode(b, layer0, n_layers, Q, q_pos, q_heads, out, splits, Knew, Vnew, early, c0->stream));
         return SVLM_OK;
     }
+    if (Knew) return SVLM_ERR_ARG;   // the fused step exists for the split-KV kernel only
     if (n_q >= 2 && svlm_prefill_supported(c0->dev.n_pages, group)) {
         SVLM_CUDA(svlm_launch_prefill(b, layer0, n_layers, Q, q_pos, n_q, q_heads, out, c0->stream));
         return SVLM_OK;
@@ -210,10 +238,12 @@ int svlm_cache_create(svlm_cache** out, int layers, int kv_heads, int head_dim, 
     A(dev_alloc(c, &d.V, slab));
     {
         unsigned char* tm = nullptr;
-        A(dev_alloc(c, &tm, 256));
+        A(dev_alloc(c, &tm, 512));
         d.tmaps = tm;
     }
+    A(dev_alloc(c, &d.rope_tab, (size_t)3 * 256 * (head_dim / 2) * 2, false));
     if (rc == SVLM_OK) rc = make_tensor_maps(c);
+    if (rc == SVLM_OK) rc = upload_rope_table(c);
     if (rc == SVLM_OK) {
         // pool pages on the free stack (top of the stack = lowest page number)
         std::vector<int> stack;
@@ -261,7 +291,8 @@ int svlm_cache_set_rope(svlm_cache* c, int mode, double base, const int sections
     }
     c->dev.rope_mode = mode;
     fill_theta(c->dev, base);
-    return SVLM_OK;
+    DeviceGuard guard(c->device);
+    return upload_rope_table(c);
 }
 
 int svlm_cache_set_policy(svlm_cache* c, int sink_any_type, int contiguous) {
@@ -282,6 +313,7 @@ int svlm_cache_append(svlm_cache* c, int layer, const void* K, const void* V, co
                       const int32_t* pos, int n) {
     if (!c || !K || !V || n < 1 || layer < -1 || layer >= c->dev.layers) return SVLM_ERR_ARG;
     DeviceGuard guard(c->device);
+    c->last_decode_layer = -1;
     if (layer <= 0) {
         if (!token_type || !pos) return SVLM_ERR_ARG;
         if (n > c->dev.capacity) return SVLM_ERR_CAPACITY;
@@ -300,6 +332,7 @@ int svlm_cache_append(svlm_cache* c, int layer, const void* K, const void* V, co
 int svlm_cache_evict(svlm_cache* c) {
     if (!c) return SVLM_ERR_ARG;
     DeviceGuard guard(c->device);
+    c->last_decode_layer = -1;
     svlm_launch_evict_meta(c->dev, c->stream);
     if (c->dev.contiguous) svlm_launch_evict_rotate(c->dev, c->stream);
     SVLM_CUDA(cudaGetLastError());
@@ -310,6 +343,25 @@ int svlm_attend(svlm_cache* c, int layer, const void* Q, const int32_t* q_pos, i
     if (!c) return SVLM_ERR_ARG;
     svlm_cache* one[1] = {c};
     return attend_common(one, 1, layer, Q, q_pos, n_q, q_heads, out);
+}
+
+int svlm_decode_step(svlm_cache* c, int layer, const void* K, const void* V, const uint8_t* token_type,
+                     const int32_t* pos, const void* Q, int q_heads, void* out) {
+    if (!c || !K || !V || !pos || !Q || !out || layer < 0 || layer >= c->dev.layers || q_heads < 1) return SVLM_ERR_ARG;
+    if (q_heads % c->dev.kv_heads || q_heads / c->dev.kv_heads > 8) return SVLM_ERR_ARG;
+    DeviceGuard guard(c->device);
+    if (layer == 0) {
+        if (!token_type) return SVLM_ERR_ARG;
+        c->configured_locked = true;
+        c->last_decode_layer = -1;
+        svlm_launch_append_meta(c->dev, token_type, pos, 1, c->stream);
+        c->appended += 1;
+        c->pending_n = 1;
+    } else if (c->pending_n != 1) {
+        return SVLM_ERR_ORDER;
+    }
+    svlm_cache* one[1] = {c};
+    return attend_common(one, 1, layer, Q, pos, 1, q_heads, out, K, V);
 }
 
 int svlm_attend_batched(svlm_cache* const* caches, int n_caches, int layer, const void* Q, const int32_t* q_pos,

@@ -79,6 +79,34 @@ class SideBySide:
     def append_decode_token(self):
         self._append(*self.stream.next_decode_token())
 
+    def decode_step_fused(self, layers=None):
+        """One generated token through svlm_decode_step, layer after layer (append and attention in one
+        launch per layer); returns the error statistics of every layer against the checker."""
+        gids, types, pos = self.stream.next_decode_token()
+        ty, ps = torch.from_numpy(types).cuda(), torch.from_numpy(np.ascontiguousarray(pos)).cuda()
+        outs, Qs = [], []
+        for l in range(self.layers):
+            Qs.append(self.stream.q(l, gids))
+            outs.append(dev_to_f64(self.cache.decode_step(l, bits_to_dev(self.stream.k(l, gids)),
+                                                          bits_to_dev(self.stream.v(l, gids)),
+                                                          ty if l == 0 else None, ps, bits_to_dev(Qs[-1]))))
+        assert self.cache.status() == binding.OK
+        self.ref.append(None, None, types, pos)
+        self.last = (gids, types, pos)
+        stats = []
+        for l in (range(self.layers) if layers is None else layers):
+            self._give_values_to_ref(l)
+            stats.append(self._stats(outs[l], self.ref.attend(l, Qs[l], pos)))
+        return stats
+
+    @staticmethod
+    def _stats(out, want):
+        err = np.abs(out - want)
+        excess = float((err - (TIGHT_ABS + TIGHT_REL * np.abs(want))).max())
+        rms_ratio = float(np.sqrt((err ** 2).mean()) / max(np.sqrt((want ** 2).mean()), 1e-30)) if want.any() else \
+            float(err.max())
+        return float(err.max()), float(err.mean()), rms_ratio, excess
+
     def evict(self):
         self.cache.evict()
         self.ref.evict()
@@ -133,11 +161,7 @@ class SideBySide:
         want = self.ref.attend(layer, Qb, pos, rows)
         if rows is not None:
             out = out[np.asarray(rows)]
-        err = np.abs(out - want)
-        excess = float((err - (TIGHT_ABS + TIGHT_REL * np.abs(want))).max())
-        rms_ratio = float(np.sqrt((err ** 2).mean()) / max(np.sqrt((want ** 2).mean()), 1e-30)) if want.any() else \
-            float(err.max())
-        return float(err.max()), float(err.mean()), rms_ratio, excess
+        return self._stats(out, want)
 
 
 def assert_close(stats, tight=True):

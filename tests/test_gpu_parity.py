@@ -28,10 +28,15 @@ def test_config1_every_output():
         st = s.attend(0)
         assert_close(st)
         worst = [max(worst[0], st[0]), max(worst[1], st[1])]
-        for _ in range(wl.decode_steps):
-            s.append_decode_token()
-            assert_close(s.attend(0))
+        for d in range(wl.decode_steps):
+            if d % 2:
+                for st in s.decode_step_fused():      # append + attention in one launch
+                    assert_close(st)
+            else:
+                s.append_decode_token()
+                assert_close(s.attend(0))
         s.check_metadata()
+        s.check_kv(0)
     print("config 1 worst max/mean abs error", worst)
 
 
@@ -50,9 +55,14 @@ def test_scaled_mrope_stream_multi_layer(sink_any, contiguous):
         layer = chunk % 3
         s.check_kv(layer)
         assert_close(s.attend(layer, all_layers=(chunk % 3 == 0)))
-        for _ in range(wl.decode_steps):
-            s.append_decode_token()
-            assert_close(s.attend((layer + 1) % 3))
+        for d in range(wl.decode_steps):
+            if (chunk + d) % 2:
+                for st in s.decode_step_fused():
+                    assert_close(st)
+            else:
+                s.append_decode_token()
+                assert_close(s.attend((layer + 1) % 3))
+        s.check_kv((layer + 2) % 3)
     s.evict()
     s.evict()      # a second evict with nothing new must change nothing
     s.check_metadata()
@@ -76,8 +86,9 @@ def test_layer_sequential_appends_after_the_evict():
             assert_close(s.attend(l))
         s.check_kv(chunk % 3)
         for _ in range(wl.decode_steps):
-            s.append_decode_token()
-            assert_close(s.attend(chunk % 3))
+            for st in s.decode_step_fused():
+                assert_close(st)
+        s.check_kv((chunk + 1) % 3)
 
 
 @pytest.mark.parametrize("S,Vw,Tw", [(0, 64, 16), (8, 0, 16), (8, 64, 0), (0, 0, 0), (300, 64, 16)])

@@ -52,11 +52,11 @@ def test_noalloc_decode_matches_regular_entry_point_twice():
 
 def test_noalloc_rejects_what_does_not_fit():
     from paper_2510_09608_b200 import binding
-    # 64 KV heads x 16 splits x (8*128+16) floats does not fit the 1 MiB array
-    cache = binding.Cache(1, 64, 128, 4, 2048, 64, 4096)
-    K = torch.zeros(1, 64, 128, dtype=torch.bfloat16, device="cuda")
+    # 256 KV heads x (8*128+16) floats of partial results do not fit the 1 MiB array
+    cache = binding.Cache(1, 256, 128, 4, 64, 32, 128)
+    K = torch.zeros(1, 256, 128, dtype=torch.bfloat16, device="cuda")
     cache.append(0, K, K, torch.zeros(1, dtype=torch.uint8, device="cuda"), torch.zeros(1, dtype=torch.int32, device="cuda"))
     with pytest.raises(binding.SvlmError) as e:
-        cache.attend_decode_noalloc(0, torch.zeros(1, 64, 128, dtype=torch.bfloat16, device="cuda"),
+        cache.attend_decode_noalloc(0, torch.zeros(1, 256, 128, dtype=torch.bfloat16, device="cuda"),
                                     torch.zeros(1, dtype=torch.int32, device="cuda"))
     assert e.value.status == binding.ERR_TOO_LARGE
