@@ -176,9 +176,9 @@ int svlm_attend_host(svlm_cache* c, int layer, const void* Q_host, const int32_t
  *   q_heads         a multiple of kv_heads, at most 8 query heads per KV head
  * Limits and rules
  *   - the array is resident on every GPU that loads the library, for the life of the process;
- *   - kv_heads x (number of KV splits: about one CTA per SM over the KV heads) x (8*head_dim + 16)
- *     floats plus one counter per (layer, kv_head) must fit in it, otherwise SVLM_ERR_TOO_LARGE is
- *     returned and nothing runs (28 layers x 4 KV heads x head_dim 128 needs about 0.6 MB);
+ *   - kv_heads x (number of KV splits: about one CTA per SM over the KV heads) x (16*head_dim + 64)
+ *     bytes plus one counter per (layer, kv_head) must fit in it, otherwise SVLM_ERR_TOO_LARGE is
+ *     returned and nothing runs (28 layers x 4 KV heads x head_dim 128 needs about 0.31 MB);
  *   - all calls on one GPU share the array and it keeps the previous call's contents; the call
  *     clears what has to start at zero, on the cache's stream, before its kernel.  Calls whose
  *     kernels can overlap on the GPU (different streams, different caches) race on it: order them;
@@ -187,7 +187,7 @@ int svlm_attend_host(svlm_cache* c, int layer, const void* Q_host, const int32_t
  * Errors: SVLM_ERR_ARG, SVLM_ERR_ORDER (nothing appended yet), SVLM_ERR_TOO_LARGE, SVLM_ERR_CUDA.
  * The result equals svlm_attend's for the same state and inputs.
  */
-#define SVLM_NOALLOC_SCRATCH_BYTES (1u << 20)
+#define SVLM_NOALLOC_SCRATCH_BYTES (512u << 10)
 int svlm_attend_decode_noalloc(svlm_cache* c, int layer, const void* Q, const int32_t* q_pos, int q_heads, void* out);
 
 /*

@@ -13,7 +13,7 @@ import numpy as np
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libsvlm.so")
+LIB_PATH = os.environ.get("SVLM_LIBRARY") or os.path.join(_HERE, "libsvlm.so")   # SVLM_LIBRARY: a library built elsewhere
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2510_09608_b200.build`; "

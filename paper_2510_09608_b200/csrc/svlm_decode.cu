@@ -35,7 +35,7 @@ namespace {
 
 using namespace svlm_ptx;
 
-constexpr int DEC_CWARPS = 4;                       // consumer warps
+constexpr int DEC_CWARPS = 8;                       // consumer warps
 constexpr int DEC_THREADS = (DEC_CWARPS + 1) * 32;  // + one producer warp
 constexpr int DEC_STAGES = 6;
 constexpr int SUB = 32;                             // keys per sub-tile
@@ -70,9 +70,13 @@ __device__ __forceinline__ unsigned pack_bf16(float lo, float hi) {
 }
 
 // Scratch layout per cache: arrival counters [layers*kv_heads] (kept at zero between launches),
-// then per (layer in launch, kv head): splits x { o[8][D], m[8], l[8] } floats.
+// then per (layer in launch, kv head): splits records { o[8][D] bf16, m[8] f32, l[8] f32 }.  The
+// un-normalised partial outputs travel as bf16 (their error is of the size of the final rounding of
+// the output), which lets the combining CTA stage every record in shared memory in one round trip.
 template <int D>
-__host__ __device__ constexpr int partial_floats() { return 8 * D + 16; }
+__host__ __device__ constexpr int rec_bytes() { return 8 * D * 2 + 64; }
+template <int D>
+__host__ __device__ constexpr int partial_floats() { return rec_bytes<D>() / 4; }
 
 struct DecShared {
     unsigned long long full[DEC_STAGES], empty[DEC_STAGES];
@@ -88,7 +92,7 @@ __device__ __forceinline__ int sw_off(int key, int chunk) {
 }
 
 template <int D>
-__global__ void __launch_bounds__(DEC_THREADS, 1)
+__global__ void __launch_bounds__(DEC_THREADS, 2)
 decode_kernel(SvlmAttendBatch b, int layer0, int n_layers, const uint16_t* __restrict__ Q,
               const int* __restrict__ q_pos, int q_heads, uint16_t* __restrict__ out, int splits,
               const uint16_t* __restrict__ Knew, const uint16_t* __restrict__ Vnew, int early_loads) {
@@ -129,6 +133,16 @@ decode_kernel(SvlmAttendBatch b, int layer0, int n_layers, const uint16_t* __res
         const int4 tl = __ldcg(reinterpret_cast<const int4*>(vw.tiles + i));   // page, lo, hi, pad
         sh.tile_pk[i] = (unsigned)tl.x | ((unsigned)tl.y << 16) | ((unsigned)tl.z << 24);
     }
+    if (early_loads && threadIdx.x < 3) {
+        // Bring the call's own small inputs towards L2 while the previous kernel still runs (a hint:
+        // they are read for real only after the grid-dependency wait).
+        const size_t qoff = ((size_t)prob * q_heads + (size_t)hk * G) * D, koff = ((size_t)prob * b.kv_heads + hk) * D;
+        const void* p = threadIdx.x == 0 ? (const void*)(Q + qoff) : threadIdx.x == 1 ? (const void*)(Knew ? Knew + koff : Q + qoff)
+                                                                                     : (const void*)(Vnew ? Vnew + koff : Q + qoff);
+        const int bytes = threadIdx.x == 0 ? G * D * 2 : D * 2;
+        for (int o = 0; o < bytes; o += 128)
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char*>(p) + o));
+    }
     const long long shift = __ldcg(&vw.ctrl->shift_total);
     // the new token of a fused step: where it lives and whether it is still stored there
     int new_slot = -1;
@@ -141,9 +155,9 @@ decode_kernel(SvlmAttendBatch b, int layer0, int n_layers, const uint16_t* __res
     const int total_q = 4 * n_tiles;
     const int q0 = (int)((long long)split * total_q / splits), q1 = (int)((long long)(split + 1) * total_q / splits);
     const size_t head_row0 = ((size_t)layer * b.kv_heads + hk) * b.n_slots;
-    const size_t part_floats = partial_floats<D>();
-    float* ws_parts = vw.ws + (((size_t)b.layers * b.kv_heads + 3) & ~(size_t)3);   // after the counters (16-byte aligned)
-    float* part = ws_parts + ((size_t)(li * b.kv_heads + hk) * splits + split) * part_floats;
+    constexpr int REC = rec_bytes<D>();
+    unsigned char* ws_parts = reinterpret_cast<unsigned char*>(vw.ws + (((size_t)b.layers * b.kv_heads + 3) & ~(size_t)3));
+    unsigned char* part = ws_parts + ((size_t)(li * b.kv_heads + hk) * splits + split) * REC;   // 16-byte aligned
 
     auto sub_valid = [&](int q, int& page, int& lo, int& hi) {
         const unsigned pk = sh.tile_pk[q >> 2];
@@ -177,15 +191,22 @@ decode_kernel(SvlmAttendBatch b, int layer0, int n_layers, const uint16_t* __res
         }
     } else {
         // ================= consumers =================
-        if (early_loads) pdl_wait();   // from here on: data that earlier kernels in the stream produced
         const float2* tab = reinterpret_cast<const float2*>(b.rope_tab);
         // ---- query rows: rotate at q_pos - shift_total, round to bf16, park in shared memory ----
         {
             const int pair = threadIdx.x & (HALF - 1);
             const int axis = b.rope_mode == 0 ? 0 : (pair < b.sec_t ? 0 : (pair < b.sec_th ? 1 : 2));
-            const int* qp = q_pos + (size_t)ci * (b.rope_mode == 0 ? 1 : 3);
-            const long long c = (long long)qp[b.rope_mode == 0 ? 0 : axis] - shift;
-            const float2 cs = svlm_rope_cs(tab, HALF, pair, c, b.theta[pair]);
+            float2 cs;
+            if (new_slot >= 0) {
+                // fused step: the query is the appended token, its position is already in the metadata,
+                // so the rotation factors do not have to wait for the previous kernel
+                cs = svlm_rope_cs(tab, HALF, pair, __ldcg(vw.slot_c + (size_t)axis * b.n_slots + new_slot), b.theta[pair]);
+                if (early_loads) pdl_wait();
+            } else {
+                if (early_loads) pdl_wait();
+                const int* qp = q_pos + (size_t)ci * (b.rope_mode == 0 ? 1 : 3);
+                cs = svlm_rope_cs(tab, HALF, pair, (long long)qp[b.rope_mode == 0 ? 0 : axis] - shift, b.theta[pair]);
+            }
             for (int h = threadIdx.x / HALF; h < 8; h += (DEC_CWARPS * 32) / HALF) {
                 float lo = 0.f, hi = 0.f;
                 if (h < G) {
@@ -333,9 +354,10 @@ decode_kernel(SvlmAttendBatch b, int layer0, int n_layers, const uint16_t* __res
             l[0] += __shfl_xor_sync(0xffffffffu, l[0], sft);
             l[1] += __shfl_xor_sync(0xffffffffu, l[1], sft);
         }
-        // ---- merge the consumer warps: s_o[warp][8 heads][D], s_m/s_l[warp][8] (own region, after s_q)
-        float* s_o = reinterpret_cast<float*>(s_q + 8 * D);
-        float* s_m = s_o + DEC_CWARPS * 8 * D;
+        // ---- merge the consumer warps through shared memory (the ring is free once all are here) ----
+        asm volatile("bar.sync 1, %0;" ::"n"(DEC_CWARPS * 32));
+        float* s_o = reinterpret_cast<float*>(ring);          // [warp][8 heads][D]
+        float* s_m = s_o + DEC_CWARPS * 8 * D;                // [warp][8]
         float* s_l = s_m + DEC_CWARPS * 8;
 #pragma unroll
         for (int db = 0; db < DBLK; ++db) {
@@ -351,29 +373,37 @@ decode_kernel(SvlmAttendBatch b, int layer0, int n_layers, const uint16_t* __res
         }
         asm volatile("bar.sync 1, %0;" ::"n"(DEC_CWARPS * 32));
         const int ct = threadIdx.x;   // 0 .. DEC_CWARPS*32-1
-        for (int i = ct; i < 8 * D; i += DEC_CWARPS * 32) {
-            const int h = i / D;
+        if (ct < D) {                 // eight consecutive output elements of one head
+            const int h = ct / (D / 8), d0 = (ct % (D / 8)) * 8;
             float M = -INFINITY;
 #pragma unroll
             for (int w = 0; w < DEC_CWARPS; ++w) M = fmaxf(M, s_m[w * 8 + h]);
-            float acc = 0.f;
+            float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
             if (M > -INFINITY)
 #pragma unroll
-                for (int w = 0; w < DEC_CWARPS; ++w) acc += s_o[(size_t)w * 8 * D + i] * exp2f(s_m[w * 8 + h] - M);
-            part[i] = acc;
-        }
-        if (ct < 8) {
-            const int h = ct;
+                for (int w = 0; w < DEC_CWARPS; ++w) {
+                    const float f = exp2f(s_m[w * 8 + h] - M);
+                    const float4 a = *reinterpret_cast<const float4*>(s_o + (size_t)w * 8 * D + h * D + d0);
+                    const float4 c = *reinterpret_cast<const float4*>(s_o + (size_t)w * 8 * D + h * D + d0 + 4);
+                    acc[0] += a.x * f; acc[1] += a.y * f; acc[2] += a.z * f; acc[3] += a.w * f;
+                    acc[4] += c.x * f; acc[5] += c.y * f; acc[6] += c.z * f; acc[7] += c.w * f;
+                }
+            uint4 pk;
+            pk.x = pack_bf16(acc[0], acc[1]); pk.y = pack_bf16(acc[2], acc[3]);
+            pk.z = pack_bf16(acc[4], acc[5]); pk.w = pack_bf16(acc[6], acc[7]);
+            *reinterpret_cast<uint4*>(part + (size_t)(h * D + d0) * 2) = pk;
+        } else if (ct < D + 8) {
+            const int h = ct - D;
             float M = -INFINITY, L = 0.f;
 #pragma unroll
             for (int w = 0; w < DEC_CWARPS; ++w) M = fmaxf(M, s_m[w * 8 + h]);
             if (M > -INFINITY)
 #pragma unroll
                 for (int w = 0; w < DEC_CWARPS; ++w) L += s_l[w * 8 + h] * exp2f(s_m[w * 8 + h] - M);
-            part[8 * D + h] = M;
-            part[8 * D + 8 + h] = L;
+            float* ml = reinterpret_cast<float*>(part + 8 * D * 2);
+            ml[h] = M;
+            ml[8 + h] = L;
         }
-        __threadfence();
     }
 
     // ---- last CTA of this (cache, layer, kv head) combines the splits -----------------------------
@@ -390,61 +420,81 @@ decode_kernel(SvlmAttendBatch b, int layer0, int n_layers, const uint16_t* __res
         __syncthreads();
         return;
     }
+    // The barrier above ordered every thread's partial-result stores before thread 0's release.
     unsigned* counter = reinterpret_cast<unsigned*>(vw.ws) + li * b.kv_heads + hk;
     if (threadIdx.x == 0) {
-        const unsigned prev = atomicAdd(counter, 1u);
+        unsigned prev;
+        asm volatile("atom.add.acq_rel.gpu.global.u32 %0, [%1], 1;" : "=r"(prev) : "l"(counter) : "memory");
         sh.last = (prev == (unsigned)splits - 1);
         if (sh.last) *counter = 0;   // ready for the next launch
     }
     __syncthreads();
     if (!sh.last) return;
-    __threadfence();
-    // Phase 1: per-split (m, l) into shared memory, then per-head global max, weights and 1/L.
-    const float* parts = ws_parts + (size_t)(li * b.kv_heads + hk) * splits * part_floats;
-    float* c_m = reinterpret_cast<float*>(ring);          // [splits][8] -> weights exp2(m - M)
-    float* c_l = c_m + splits * 8;                        // [splits][8]
-    float* c_inv = c_l + splits * 8;                      // [8]
-    for (int i = threadIdx.x; i < splits * 16; i += DEC_THREADS) {
-        const int sp = i >> 4, j = i & 15;
-        const float v = __ldcg(parts + (size_t)sp * part_floats + 8 * D + j);
-        (j < 8 ? c_m : c_l)[sp * 8 + (j & 7)] = v;
-    }
-    __syncthreads();
-    if (threadIdx.x < 8) {
-        const int h = threadIdx.x;
-        float M = -INFINITY, L = 0.f;
-        for (int sp = 0; sp < splits; ++sp) M = fmaxf(M, c_m[sp * 8 + h]);
-        for (int sp = 0; sp < splits; ++sp) {
-            const float f = M > -INFINITY ? exp2f(c_m[sp * 8 + h] - M) : 0.f;
-            c_m[sp * 8 + h] = f;
-            L += c_l[sp * 8 + h] * f;
+    // Stage the splits' records in shared memory with independent 16-byte loads by every thread (one
+    // round trip to L2 for as many records as fit, normally all), then two threads per group of eight
+    // output elements merge them (even and odd records) and add up through a shuffle.
+    const unsigned char* parts = ws_parts + (size_t)(li * b.kv_heads + hk) * splits * REC;
+    constexpr int PER_ROUND = DEC_STAGES * STAGE_BYTES / REC;
+    const int pairs = G * (D / 8);                      // groups of eight output elements
+    const int grp = threadIdx.x >> 1, sub = threadIdx.x & 1;
+    const bool owner = grp < pairs;
+    const int h = grp / (D / 8), d0 = (grp % (D / 8)) * 8;
+    float M = -INFINITY, L = 0.f;
+    float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    for (int sp0 = 0; sp0 < splits; sp0 += PER_ROUND) {
+        const int n = min(PER_ROUND, splits - sp0);
+        __syncthreads();   // the ring is free (first round: merge buffers; later: previous round read)
+        {
+            // asynchronous 16-byte copies straight into shared memory: no registers, all in flight at once
+            const unsigned char* src = parts + (size_t)sp0 * REC;
+            const int n16 = n * (REC / 16);
+            for (int i = threadIdx.x; i < n16; i += DEC_THREADS)
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(ring + (size_t)i * 16)),
+                             "l"(src + (size_t)i * 16) : "memory");
+            asm volatile("cp.async.commit_group;" ::: "memory");
+            asm volatile("cp.async.wait_group 0;" ::: "memory");
         }
-        c_inv[h] = L > 0.f ? 1.f / L : 0.f;
-    }
-    __syncthreads();
-    // Phase 2: weighted sum of the split outputs; all loads of a thread are independent.
-    for (int i0 = 0; i0 < 8 * D; i0 += DEC_THREADS * 4) {
-        const int i = i0 + threadIdx.x * 4;
-        if (i >= G * D) continue;
-        const int h = i / D;
-        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int sp = 0; sp < splits; ++sp) {
-            const float4 v = __ldcg(reinterpret_cast<const float4*>(parts + (size_t)sp * part_floats + i));
-            const float w = c_m[sp * 8 + h];
-            acc.x += v.x * w; acc.y += v.y * w; acc.z += v.z * w; acc.w += v.w * w;
+        __syncthreads();
+        if (owner) {
+            float bm = -INFINITY;
+            for (int r = 0; r < n; ++r) bm = fmaxf(bm, *reinterpret_cast<const float*>(ring + (size_t)r * REC + 8 * D * 2 + h * 4));
+            const float Mn = fmaxf(M, bm);
+            if (Mn > -INFINITY) {
+                const float resc = exp2f(M - Mn);   // M = -inf gives 0
+                L *= resc;
+#pragma unroll
+                for (int e = 0; e < 8; ++e) acc[e] *= resc;
+#pragma unroll 4
+                for (int r = sub; r < n; r += 2) {
+                    const unsigned char* rec = ring + (size_t)r * REC;
+                    const float w = exp2f(*reinterpret_cast<const float*>(rec + 8 * D * 2 + h * 4) - Mn);
+                    L += *reinterpret_cast<const float*>(rec + 8 * D * 2 + 32 + h * 4) * w;
+                    const uint4 v = *reinterpret_cast<const uint4*>(rec + (size_t)(h * D + d0) * 2);
+                    acc[0] += __uint_as_float(v.x << 16) * w; acc[1] += __uint_as_float(v.x & 0xffff0000u) * w;
+                    acc[2] += __uint_as_float(v.y << 16) * w; acc[3] += __uint_as_float(v.y & 0xffff0000u) * w;
+                    acc[4] += __uint_as_float(v.z << 16) * w; acc[5] += __uint_as_float(v.z & 0xffff0000u) * w;
+                    acc[6] += __uint_as_float(v.w << 16) * w; acc[7] += __uint_as_float(v.w & 0xffff0000u) * w;
+                }
+                M = Mn;
+            }
         }
-        const float inv = c_inv[h];
-        uint2 pk;
-        pk.x = pack_bf16(acc.x * inv, acc.y * inv);
-        pk.y = pack_bf16(acc.z * inv, acc.w * inv);
-        *reinterpret_cast<uint2*>(out + ((size_t)prob * q_heads + hk * G + h) * D + (i % D)) = pk;
+    }
+    // even + odd records (both threads of a pair used the same maximum)
+    L += __shfl_xor_sync(0xffffffffu, L, 1);
+#pragma unroll
+    for (int e = 0; e < 8; ++e) acc[e] += __shfl_xor_sync(0xffffffffu, acc[e], 1);
+    if (owner && sub == 0) {
+        const float inv = L > 0.f ? 1.f / L : 0.f;
+        uint4 pk;
+        pk.x = pack_bf16(acc[0] * inv, acc[1] * inv); pk.y = pack_bf16(acc[2] * inv, acc[3] * inv);
+        pk.z = pack_bf16(acc[4] * inv, acc[5] * inv); pk.w = pack_bf16(acc[6] * inv, acc[7] * inv);
+        *reinterpret_cast<uint4*>(out + ((size_t)prob * q_heads + hk * G + h) * D + d0) = pk;
     }
 }
 
 template <int D>
 constexpr size_t decode_smem() {
-    return sizeof(DecShared) + 1024 + (size_t)DEC_STAGES * 2 * SUB * D * 2 + 8 * D * 2 +
-           (size_t)DEC_CWARPS * 8 * D * 4 + DEC_CWARPS * 16 * 4;
+    return sizeof(DecShared) + 1024 + (size_t)DEC_STAGES * 2 * SUB * D * 2 + 8 * D * 2;
 }
 
 }  // namespace

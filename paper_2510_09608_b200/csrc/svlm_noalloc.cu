@@ -8,7 +8,7 @@
 // are not permitted at all.  The regular path sizes its scratch when the cache is created; this one
 // works with any cache, including one whose creator gave it no scratch, because it brings its own.
 //
-// The array lives in every GPU that loads the library until the process exits (1 MiB per device).
+// The array lives in every GPU that loads the library until the process exits (512 KiB per device).
 // All calls on a device share it, and it keeps whatever the previous call left behind: the arrival
 // counters are cleared on the stream before every launch, the partial results are fully rewritten
 // before they are read.  Two calls whose kernels overlap on the GPU (different streams) would race
