@@ -2,76 +2,67 @@
 // retained cache plus, causally, the chunk itself (paper Section 2.1: the retained KV is reused, only
 // the new second of tokens is computed).  This is the one dense contraction of the path, so it runs
 // on the 5th-generation tensor cores:
-//   * the G query heads that share a KV head are packed along M (row = (token, head-in-group)), so a
-//     128-row tile reads each key/value tile once for the whole group;
-//   * K and V tiles (one 128-slot page each) arrive by TMA (128-byte swizzle) into a 2-stage ring;
-//   * S = Q K^T is issued by one thread with tcgen05.mma into one of two 128-column TMEM buffers, so
-//     the tensor core computes tile j+1 while the softmax warps work on tile j;
-//   * four softmax warps (one thread per row) read S with tcgen05.ld, keep a lazily updated running
-//     maximum (O is rescaled only when the maximum grows by more than 2^8), write P as bf16 into
-//     swizzled shared memory, and O += P V accumulates in TMEM (V is the MN-major B operand);
-//   * causal and partial-page masking only touches the few tiles that hold new-chunk tokens or a
-//     ring's ragged end; whole tiles that no row of the CTA may see are skipped.
-// Every wait is bounded: on expiry the CTA records SVLM_ERR_TIMEOUT in the cache's status word,
-// drains its outstanding copies, frees its TMEM and returns.
+//   * the G query heads that share a KV head are packed along M (row = (token, head-in-group));
+//   * a CTA owns 256 such rows as two 128-row tiles A and B.  Both tiles use every K/V page the CTA
+//     streams, which halves the bytes per flop that have to come out of L2 (with 128 rows per CTA
+//     the K/V stream alone took as long as the whole kernel should);
+//   * the K/V pages of one (tile pair, KV head) are split between the two CTAs of a thread-block
+//     cluster; at the end each CTA hands the un-normalised result of one tile to the other through
+//     distributed shared memory and merges and writes the tile it keeps;
+//   * K and V pages (128 slots) arrive by TMA (128-byte swizzle) into one 5-stage ring, K(j) V(j)
+//     K(j+1) ..., in the order the tensor pipe consumes them;
+//   * one thread issues tcgen05.mma: S_A, S_B = Q K^T into two 128-column TMEM buffers, O_A, O_B += P V
+//     into two TMEM accumulators, in the order PV_A(j) S_A(j+1) PV_B(j) S_B(j+1), so the tensor
+//     pipe works for one tile while the other tile's softmax warpgroup exponentiates;
+//   * two softmax warpgroups (one thread per row) read S with tcgen05.ld in 32-column chunks (a first
+//     pass for the row maximum, a second for the exponentials, the next chunk always in flight),
+//     write P as bf16 back into the TMEM columns of S, where it is the A operand of P V (no
+//     shared-memory round trip); the running maximum moves lazily (O is rescaled only when the
+//     maximum grows by more than 2^8);
+//   * rotation factors of the queries come from a table; causal and partial-page masking only
+//     touches the few pages that hold new-chunk tokens or a ring's ragged end; pages that no row
+//     of the CTA may see are skipped.
+// Every mbarrier wait is bounded: on expiry the CTA records SVLM_ERR_TIMEOUT in the cache's status
+// word, drains its outstanding copies, frees its TMEM and returns (both CTAs of a cluster still meet
+// at the hardware cluster barriers, which every thread reaches on every path).
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include "svlm_dev.h"
 #include "svlm_launch.h"
+#include "svlm_ptx.cuh"
+#include "svlm_rope.cuh"
 
 namespace {
 
-constexpr int PF_THREADS = 192;       // warps 0-3 softmax/epilogue, warp 4 TMA, warp 5 MMA issue
-constexpr int PF_STAGES = 2;
+using namespace svlm_ptx;
+
+#ifndef PF_ISSUERS
+#define PF_ISSUERS 1                  // threads that issue tcgen05.mma (two interleaving streams measured slower)
+#endif
+constexpr int PF_THREADS = 288 + 32 * PF_ISSUERS;   // warps 0-3: softmax of tile A, 4-7: tile B; warp 8: TMA; warp 9 (, 10): MMA issue
+constexpr int PF_RING = 5;            // K/V page stages
 constexpr int PF_MAX_TILES = 512;
-constexpr unsigned WAIT_LIMIT = 1u << 20;
+constexpr int PF_ROWS = 256;          // rows per CTA
 
-// ---- PTX wrappers ----------------------------------------------------------------------------
-__device__ __forceinline__ unsigned smem_u32(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(void* bar, unsigned count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
-}
-__device__ __forceinline__ void mbar_arrive(void* bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(void* bar, unsigned bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_test(void* bar, unsigned parity) {
-    unsigned ok;
-    asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
-                 : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
-    return ok != 0;
-}
-// Bounded wait: false when the limit ran out or another thread of the CTA already gave up.
-__device__ __forceinline__ bool mbar_wait(void* bar, unsigned parity, volatile int* abort_flag) {
-    for (unsigned it = 0; it < WAIT_LIMIT; ++it) {
-        if (mbar_test(bar, parity)) return true;
-        if ((it & 63) == 63) {
-            if (*abort_flag) return false;
-            __nanosleep(64);
-        }
-    }
-    *abort_flag = 1;
-    return false;
-}
-__device__ __forceinline__ void tma_load_2d(void* dst, const void* tmap, int x, int y, void* bar) {
-    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-                 ::"r"(smem_u32(dst)), "l"(tmap), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(void* bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
-__device__ __forceinline__ void tc_mma(unsigned d_tmem, unsigned long long a_desc, unsigned long long b_desc,
-                                       unsigned idesc, unsigned accumulate) {
+// D[tmem] (+)= A[smem] * B[smem]
+__device__ __forceinline__ void tc_mma_ss(unsigned d_tmem, unsigned long long a_desc, unsigned long long b_desc,
+                                          unsigned idesc, unsigned accumulate) {
     asm volatile("{\n.reg .pred p;\nsetp.ne.u32 p, %4, 0;\n"
                  "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
                  ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem]
+__device__ __forceinline__ void tc_mma_ts(unsigned d_tmem, unsigned a_tmem, unsigned long long b_desc, unsigned idesc,
+                                          unsigned accumulate) {
+    asm volatile("{\n.reg .pred p;\nsetp.ne.u32 p, %4, 0;\n"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}"
+                 ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
 __device__ __forceinline__ void tmem_ld32(unsigned taddr, float* v) {
     unsigned* r = reinterpret_cast<unsigned*>(v);
@@ -95,8 +86,37 @@ __device__ __forceinline__ void tmem_st32(unsigned taddr, const float* v) {
                    "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
                  : "memory");
 }
+__device__ __forceinline__ void tmem_st16(unsigned taddr, const unsigned* r) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+                 "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
+                 ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+                   "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+                 : "memory");
+}
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// Hardware barrier of the thread-block cluster (every thread of both CTAs takes part).
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\nbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ unsigned cluster_rank() {
+    unsigned r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// Address of this CTA's shared-memory location `p` as seen in CTA `rank` of the cluster.
+__device__ __forceinline__ unsigned map_to_rank(const void* p, unsigned rank) {
+    unsigned a;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(a) : "r"(smem_u32(p)), "r"(rank));
+    return a;
+}
+__device__ __forceinline__ void st_cluster_v4(unsigned addr, float4 v) {
+    asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
+}
+__device__ __forceinline__ void st_cluster_v2(unsigned addr, float2 v) {
+    asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};" ::"r"(addr), "f"(v.x), "f"(v.y) : "memory");
+}
 
 // Shared-memory matrix descriptor, 128-byte swizzle, version 1 (sm_100).  Offsets in bytes.
 __device__ __forceinline__ unsigned long long smem_desc(unsigned addr, unsigned lbo, unsigned sbo) {
@@ -114,29 +134,111 @@ __device__ __forceinline__ unsigned pack2(float a, float b) {
     return *reinterpret_cast<unsigned*>(&v);
 }
 
+__device__ __forceinline__ float ex2(float x) {
+    float y;
+    asm volatile("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// One page of one row: S (128 fp32 columns at tS, this thread's TMEM lane) -> P (bf16 pairs in the first 64
+// columns of the same buffer), with the lazily moving reference maximum.  Two passes over S in halves of
+// 64 columns (two 32-column loads in flight at a time): row maximum, then exponentials.  P chunk ch
+// (16 columns) lands where S columns [16 ch, 16 ch + 16) were; those have been read by then and the
+// loads still in flight lie beyond them.  On MASKED pages the row sees the columns [vlo, vlo + vlen): stream
+// ordinals grow with the offset inside a page, so the valid and causally visible columns of a row are one interval.
+template <bool MASKED>
+__device__ __noinline__ void softmax_page(unsigned tS, unsigned tO, int D, unsigned vlo, unsigned vlen,
+                                             float c, float m_ref, bool have_o, float& rowsum, float& corr, float& m_new) {
+    auto visible = [&](int k) { return (unsigned)k - vlo < vlen; };
+    float ca[32], cb[32];
+    // ---- pass 1: row maximum
+    float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+    for (int hf = 0; hf < 2; ++hf) {
+        tmem_ld32(tS + hf * 64, ca);
+        tmem_ld32(tS + hf * 64 + 32, cb);
+        tmem_wait_ld();
+#pragma unroll
+        for (int k = 0; k < 32; ++k) {
+            const float a = MASKED ? (visible(hf * 64 + k) ? ca[k] : -INFINITY) : ca[k];
+            const float bq = MASKED ? (visible(hf * 64 + 32 + k) ? cb[k] : -INFINITY) : cb[k];
+            mx4[k & 3] = fmaxf(mx4[k & 3], fmaxf(a, bq));
+        }
+    }
+    tmem_ld32(tS, ca);            // first half again, for pass 2
+    tmem_ld32(tS + 32, cb);
+    const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * c;
+    // lazy running maximum: only move the reference when it would be exceeded by 2^8
+    const bool grow = mx > m_ref + 8.f;
+    m_new = grow ? mx : m_ref;
+    const float m_use = m_new == -INFINITY ? 0.f : m_new;
+    corr = grow ? exp2f(m_ref - m_use) : 1.f;   // m_ref = -inf gives 0
+    tmem_wait_ld();
+    if (have_o && __any_sync(0xffffffffu, grow)) {
+        // S of this page was issued after P V of the previous one: O is quiescent
+#pragma unroll 1
+        for (int q4 = 0; q4 < D / 32; ++q4) {
+            float o[32];
+            tmem_ld32(tO + q4 * 32, o);
+            tmem_wait_ld();
+#pragma unroll
+            for (int k = 0; k < 32; ++k) o[k] *= corr;
+            tmem_st32(tO + q4 * 32, o);
+        }
+    }
+    // ---- pass 2: exponentials in stages (all scale-subtracts, all ex2, then sums and packing), so
+    //      that the special-function pipe always has independent work queued
+    float rs4[4] = {0.f, 0.f, 0.f, 0.f};
+    auto exp_chunk = [&](float* x, int ch) {
+#pragma unroll
+        for (int k = 0; k < 32; ++k) x[k] = fmaf(x[k], c, -m_use);
+#pragma unroll
+        for (int k = 0; k < 32; ++k) x[k] = ex2(x[k]);
+        if (MASKED) {
+#pragma unroll
+            for (int k = 0; k < 32; ++k) x[k] = visible(ch * 32 + k) ? x[k] : 0.f;
+        }
+        unsigned pk[16];
+#pragma unroll
+        for (int k = 0; k < 16; ++k) {
+            rs4[k & 3] += x[2 * k] + x[2 * k + 1];
+            pk[k] = pack2(x[2 * k], x[2 * k + 1]);
+        }
+        tmem_st16(tS + ch * 16, pk);
+    };
+    exp_chunk(ca, 0);
+    exp_chunk(cb, 1);
+    tmem_ld32(tS + 64, ca);       // columns 64..127 are untouched by P (columns 0..63)
+    tmem_ld32(tS + 96, cb);
+    tmem_wait_ld();
+    exp_chunk(ca, 2);
+    exp_chunk(cb, 3);
+    rowsum = (rs4[0] + rs4[1]) + (rs4[2] + rs4[3]);
+}
+
 struct PfShared {            // control part of shared memory (tiles follow, 1024-byte aligned)
-    unsigned long long k_full[PF_STAGES], k_empty[PF_STAGES], v_full[PF_STAGES], v_empty[PF_STAGES];
-    unsigned long long s_full[2], s_empty[2], p_full, pv_done, mask_bar;
+    unsigned long long full[PF_RING], empty[PF_RING];
+    unsigned long long s_full[2], p_full[2], all_done;
     unsigned tmem_base;
     int abort_flag;
-    int tile[PF_MAX_TILES];  // page | mask<<29 | skip<<30
-    int minrow[2][SVLM_PAGE];
+    unsigned short tile[PF_MAX_TILES];     // page | mask << 14 | skip << 15
+    unsigned short minrow[2][SVLM_PAGE];   // per softmax group: first query token that may see the column
 };
+static_assert(sizeof(PfShared) <= 2040, "control block must leave room for the tiles");
 
 template <int D>
 __global__ void __launch_bounds__(PF_THREADS, 1)
 prefill_kernel(SvlmAttendBatch b, int layer0, int n_layers, const uint16_t* __restrict__ Q,
                const int* __restrict__ q_pos, int n_q, int q_heads, uint16_t* __restrict__ out) {
     constexpr int KB = D / 64;                 // 64-element (128-byte) blocks along d
-    constexpr int TILE_BYTES = 128 * D * 2;    // one K or V page of one head
+    constexpr int TILE_BYTES = 128 * D * 2;    // one K or V page of one head, or one 128-row Q tile
+    constexpr int HALF = D / 2;
     extern __shared__ unsigned char smem_raw[];
     PfShared& sh = *reinterpret_cast<PfShared*>(smem_raw);
     unsigned char* tiles_base = reinterpret_cast<unsigned char*>(
         (reinterpret_cast<uintptr_t>(smem_raw) + sizeof(PfShared) + 1023) & ~(uintptr_t)1023);
-    unsigned char* sQ = tiles_base;                           // [KB][128 rows][128 B]
-    unsigned char* sK = sQ + TILE_BYTES;                      // [stage][KB][128 keys][128 B]
-    unsigned char* sV = sK + PF_STAGES * TILE_BYTES;          // [stage][KB][128 keys][128 B]
-    unsigned char* sP = sV + PF_STAGES * TILE_BYTES;          // [2][128 rows][128 B] (keys 0-63, 64-127)
+    unsigned char* sQ = tiles_base;                           // [2 tiles][KB][128 rows][128 B]
+    unsigned char* ring = sQ + 2 * TILE_BYTES;                // [stage][KB][128 keys][128 B]
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int G = q_heads / b.kv_heads;
@@ -146,57 +248,103 @@ prefill_kernel(SvlmAttendBatch b, int layer0, int n_layers, const uint16_t* __re
     const int layer = layer0 + li;
     const SvlmAttendView& vw = b.view[ci];
     const int m_total = n_q * G;
-    const int m0 = blockIdx.x * 128;
-    const int r_lo = m0 / G, r_hi = min(n_q - 1, (m0 + 127) / G);
+    const unsigned rank = cluster_rank();      // which half of the pages this CTA takes
+    const int m0 = (blockIdx.x >> 1) * PF_ROWS;
+    const int r_lo = m0 / G, r_hi = min(n_q - 1, (m0 + PF_ROWS - 1) / G);
 
     const int n_tiles = min(vw.ctrl->n_tiles, PF_MAX_TILES);
     const long long gid_q0 = vw.ctrl->n_total - n_q;
     const long long shift = vw.ctrl->shift_total;
 
-    // ---- set-up: barriers, TMEM, tile list ------------------------------------------------------
+    // ---- set-up: barriers, TMEM, page list ------------------------------------------------------
     if (threadIdx.x == 0) {
-        for (int s = 0; s < PF_STAGES; ++s) {
-            mbar_init(&sh.k_full[s], 1); mbar_init(&sh.k_empty[s], 1);
-            mbar_init(&sh.v_full[s], 1); mbar_init(&sh.v_empty[s], 1);
-        }
-        for (int s = 0; s < 2; ++s) { mbar_init(&sh.s_full[s], 1); mbar_init(&sh.s_empty[s], 128); }
-        mbar_init(&sh.p_full, 128);
-        mbar_init(&sh.pv_done, 1);
-        mbar_init(&sh.mask_bar, 128);
+        for (int s = 0; s < PF_RING; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], PF_ISSUERS); }   // every issuer releases a page
+        for (int s = 0; s < 2; ++s) { mbar_init(&sh.s_full[s], 1); mbar_init(&sh.p_full[s], 128); }
+        mbar_init(&sh.all_done, PF_ISSUERS);
         sh.abort_flag = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        mbar_init_fence();
     }
     for (int i = threadIdx.x; i < n_tiles; i += PF_THREADS) {
         const SvlmTile tl = vw.tiles[i];
         const int skip = tl.min_gid > gid_q0 + r_hi;
         const int mask = tl.lo > 0 || tl.hi < SVLM_PAGE || tl.max_gid > gid_q0 + r_lo;
-        sh.tile[i] = tl.page | (mask << 29) | (skip << 30);
+        sh.tile[i] = (unsigned short)(tl.page | (mask << 14) | (skip << 15));
     }
-    if (warp == 4) {
+    if (warp == 8) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh.tmem_base)), "r"(512));
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
     }
 
-    // ---- query tile: rotate at q_pos - shift_total, round to bf16, store K-major swizzled ---------
-    if (warp < 4) {
-        const int m = threadIdx.x;                 // row of the tile
-        const int mg = m0 + m;
+    __syncthreads();   // barriers and page list are ready: the producer may start
+
+    const size_t head_row0 = ((size_t)layer * b.kv_heads + hk) * b.n_slots;
+    // this CTA's share of the processed pages: [p0, p1) of the non-skipped ones
+    int n_all = 0;
+    for (int j = 0; j < n_tiles; ++j) n_all += !(sh.tile[j] >> 15);
+    const int half = (n_all + 1) / 2;
+    const int p0 = rank == 0 ? 0 : half, p1 = rank == 0 ? half : n_all;
+    const int n_proc = p1 - p0;
+    volatile int* abort_flag = &sh.abort_flag;
+
+    // K/V producer state (warp 8, lane 0); the first PF_RING - 2 loads go out before the query prologue,
+    // the last two stages are borrowed by the prologue for the rotation factors
+    int pr_j = 0, pr_pi = 0, pr_n = 0;
+    bool pr_ok = true;
+    auto produce = [&](int limit) {   // issue loads until `limit` ring items have been issued in total
+        const void* tmK = vw.tmaps;
+        const void* tmV = reinterpret_cast<const unsigned char*>(vw.tmaps) + 128;
+        while (pr_ok && pr_n < limit && pr_j < n_tiles) {
+            const unsigned t = sh.tile[pr_j];
+            if (t >> 15) { ++pr_j; continue; }
+            if (pr_pi < p0 || pr_pi >= p1) { ++pr_pi; ++pr_j; continue; }
+            const int y = (int)(head_row0 + (size_t)(t & 0x3FFF) * SVLM_PAGE);
+            const int kv = pr_n & 1;      // even items are K pages, odd items V pages of the same page
+            const int st = pr_n % PF_RING;
+            pr_ok = mbar_wait(&sh.empty[st], ((pr_n / PF_RING) & 1) ^ 1, abort_flag);   // first pass: already free
+            if (!pr_ok) break;
+            mbar_expect_tx(&sh.full[st], TILE_BYTES);
+#pragma unroll
+            for (int kb = 0; kb < KB; ++kb)
+                tma_load_2d(ring + st * TILE_BYTES + kb * (128 * 128), kv ? tmV : tmK, kb * 64, y, &sh.full[st]);
+            ++pr_n;
+            if (kv) { ++pr_pi; ++pr_j; }
+        }
+    };
+    if (warp == 8 && lane == 0) produce(PF_RING - 2);
+
+    // ---- query tiles: rotate at q_pos - shift_total, round to bf16, store K-major swizzled -------
+    // (1) rotation factors of the CTA's tokens, all threads: [token][pair] (cos, sin) in the last two ring
+    //     stages (the rows of a token's G heads share them); with few heads per KV head there are too many
+    //     tokens for that space and every thread looks its own factors up instead
+    float2* s_cs = reinterpret_cast<float2*>(ring + (PF_RING - 2) * TILE_BYTES);
+    const float2* tab = reinterpret_cast<const float2*>(b.rope_tab);
+    const int n_tok = r_hi - r_lo + 1;
+    const bool cs_shared = (size_t)n_tok * HALF * sizeof(float2) <= (size_t)2 * TILE_BYTES;
+    if (cs_shared) {
+        for (int i = threadIdx.x; i < n_tok * HALF; i += PF_THREADS) {
+            const int tk = i / HALF, pair = i % HALF;
+            const int axis = b.rope_mode == 0 ? 0 : (pair < b.sec_t ? 0 : (pair < b.sec_th ? 1 : 2));
+            const int* qp = q_pos + ((size_t)ci * n_q + r_lo + tk) * (b.rope_mode == 0 ? 1 : 3);
+            s_cs[i] = svlm_rope_cs(tab, HALF, pair, (long long)qp[b.rope_mode == 0 ? 0 : axis] - shift, b.theta[pair]);
+        }
+    }
+    __syncthreads();
+    // (2) every softmax thread rotates its own row
+    if (warp < 8) {
+        const int g = warp >> 2, m = threadIdx.x & 127;
+        const int mg = m0 + g * 128 + m;
         const bool live = mg < m_total;
-        const int r = live ? mg / G : 0, h = live ? mg % G : 0;
+        const int r = live ? mg / G : r_lo, h = live ? mg % G : 0;
         const uint16_t* src = Q + ((((size_t)prob) * n_q + r) * q_heads + hk * G + h) * D;
+        const float2* cs_row = s_cs + (size_t)(r - r_lo) * HALF;
         const int* qp = q_pos + ((size_t)ci * n_q + r) * (b.rope_mode == 0 ? 1 : 3);
-        long long c3[3];
-        c3[0] = (long long)qp[0] - shift;
-        c3[1] = b.rope_mode == 0 ? c3[0] : (long long)qp[1] - shift;
-        c3[2] = b.rope_mode == 0 ? c3[0] : (long long)qp[2] - shift;
-        constexpr int HALF = D / 2;
-#pragma unroll 1
+        unsigned char* sQg = sQ + g * TILE_BYTES;
+        uint4 rowv[D / 8];                         // the whole row: every load in flight before the first use
+#pragma unroll
+        for (int i = 0; i < D / 8; ++i) rowv[i] = live ? __ldg(reinterpret_cast<const uint4*>(src) + i) : make_uint4(0, 0, 0, 0);
+#pragma unroll
         for (int c8 = 0; c8 < HALF / 8; ++c8) {    // 8 pairs at a time: chunk c8 of the low half, same of the high half
-            uint4 lo4 = make_uint4(0, 0, 0, 0), hi4 = make_uint4(0, 0, 0, 0);
-            if (live) {
-                lo4 = *reinterpret_cast<const uint4*>(src + c8 * 8);
-                hi4 = *reinterpret_cast<const uint4*>(src + HALF + c8 * 8);
-            }
+            const uint4 lo4 = rowv[c8], hi4 = rowv[HALF / 8 + c8];
             const unsigned* lw = reinterpret_cast<const unsigned*>(&lo4);
             const unsigned* hw = reinterpret_cast<const unsigned*>(&hi4);
             unsigned lo_o[4], hi_o[4];
@@ -208,225 +356,222 @@ prefill_kernel(SvlmAttendBatch b, int layer0, int n_layers, const uint16_t* __re
 #pragma unroll
                 for (int e = 0; e < 2; ++e) {
                     const int pair = c8 * 8 + 2 * j + e;
-                    const int axis = b.rope_mode == 0 ? 0 : (pair < b.sec_t ? 0 : (pair < b.sec_th ? 1 : 2));
-                    double sn, cs;
-                    sincos((double)c3[axis] * b.theta[pair], &sn, &cs);
-                    ol[e] = xl[e] * (float)cs - xh[e] * (float)sn;
-                    oh[e] = xh[e] * (float)cs + xl[e] * (float)sn;
+                    float2 cs;
+                    if (cs_shared) {
+                        cs = cs_row[pair];
+                    } else {
+                        const int axis = b.rope_mode == 0 ? 0 : (pair < b.sec_t ? 0 : (pair < b.sec_th ? 1 : 2));
+                        cs = svlm_rope_cs(tab, HALF, pair, (long long)qp[b.rope_mode == 0 ? 0 : axis] - shift, b.theta[pair]);
+                    }
+                    ol[e] = xl[e] * cs.x - xh[e] * cs.y;
+                    oh[e] = xh[e] * cs.x + xl[e] * cs.y;
                 }
                 lo_o[j] = pack2(ol[0], ol[1]);
                 hi_o[j] = pack2(oh[0], oh[1]);
             }
             // element e of the row lives in block e/64, 16-byte chunk (e%64)/8, XOR-swizzled by row&7
             const int e_lo = c8 * 8, e_hi = HALF + c8 * 8;
-            unsigned char* dl = sQ + (e_lo / 64) * (128 * 128) + m * 128 + ((((e_lo % 64) / 8) ^ (m & 7)) << 4);
-            unsigned char* dh = sQ + (e_hi / 64) * (128 * 128) + m * 128 + ((((e_hi % 64) / 8) ^ (m & 7)) << 4);
+            unsigned char* dl = sQg + (e_lo / 64) * (128 * 128) + m * 128 + ((((e_lo % 64) / 8) ^ (m & 7)) << 4);
+            unsigned char* dh = sQg + (e_hi / 64) * (128 * 128) + m * 128 + ((((e_hi % 64) / 8) ^ (m & 7)) << 4);
             *reinterpret_cast<uint4*>(dl) = make_uint4(lo_o[0], lo_o[1], lo_o[2], lo_o[3]);
             *reinterpret_cast<uint4*>(dh) = make_uint4(hi_o[0], hi_o[1], hi_o[2], hi_o[3]);
         }
-        fence_proxy_async();
     }
+    fence_proxy_async();   // the query tiles feed the tensor core, the borrowed ring stages get TMA writes next
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const unsigned tmem = sh.tmem_base;
-    const unsigned tmem_S[2] = {tmem, tmem + 128};
-    const unsigned tmem_O = tmem + 256;
-    volatile int* abort_flag = &sh.abort_flag;
+    // tile g: S (then P as bf16 pairs in its first 64 columns) at columns 128 g, O at 256 + 128 g
 
-    const size_t head_row0 = ((size_t)layer * b.kv_heads + hk) * b.n_slots;
-
-    if (warp == 4) {
-        // ================= TMA producer =================
-        if (lane == 0) {
-            const void* tmK = vw.tmaps;
-            const void* tmV = reinterpret_cast<const unsigned char*>(vw.tmaps) + 128;
-            int it = 0;
-            bool ok = true;
-            for (int j = 0; j < n_tiles && ok; ++j) {
-                const int t = sh.tile[j];
-                if (t & (1 << 30)) continue;
-                const int st = it % PF_STAGES;
-                const unsigned par = ((it / PF_STAGES) & 1) ^ 1;      // first pass over a stage: already free
-                const int y = (int)(head_row0 + (size_t)(t & 0xFFFFF) * SVLM_PAGE);
-                ok = mbar_wait(&sh.k_empty[st], par, abort_flag);
-                if (!ok) break;
-                mbar_expect_tx(&sh.k_full[st], TILE_BYTES);
-#pragma unroll
-                for (int kb = 0; kb < KB; ++kb)
-                    tma_load_2d(sK + st * TILE_BYTES + kb * (128 * 128), tmK, kb * 64, y, &sh.k_full[st]);
-                ok = mbar_wait(&sh.v_empty[st], par, abort_flag);
-                if (!ok) break;
-                mbar_expect_tx(&sh.v_full[st], TILE_BYTES);
-#pragma unroll
-                for (int kb = 0; kb < KB; ++kb)
-                    tma_load_2d(sV + st * TILE_BYTES + kb * (128 * 128), tmV, kb * 64, y, &sh.v_full[st]);
-                ++it;
-            }
-        }
-    } else if (warp == 5) {
-        // ================= MMA issuer =================
-        if (lane == 0) {
+    if (warp == 8) {
+        // ================= TMA producer: K(0) V(0) K(1) V(1) ... through one ring =================
+        if (lane == 0) produce(0x7fffffff);
+        __syncwarp();
+    } else if (warp >= 9) {
+        // ================= MMA issuers: warp 9 for tile A, warp 10 for tile B =================
+        // Per tile the order is S(0) | PV(j) S(j+1) | ...: the tensor pipe executes one thread's instructions in
+        // order, so S(j+1) overwrites the columns of P(j) only after PV(j) has read them.  Two issuing threads keep
+        // the pipe fed while one of them sits in a wait.
+        if (lane == 0 && warp - 9 < PF_ISSUERS) {
+            const int g0 = warp - 9;
             constexpr unsigned IDESC_S = make_idesc(128, 128, 0);
             constexpr unsigned IDESC_O = make_idesc(128, D, 1);
-            const unsigned q_addr = smem_u32(sQ), k_addr = smem_u32(sK), v_addr = smem_u32(sV), p_addr = smem_u32(sP);
-            auto issue_S = [&](int it) {        // S[it%2] = Q K^T for the it-th processed tile
-                const int st = it % PF_STAGES;
-                if (!mbar_wait(&sh.k_full[st], (it / PF_STAGES) & 1, abort_flag)) return false;
-                if (!mbar_wait(&sh.s_empty[it & 1], ((it >> 1) & 1) ^ 1, abort_flag)) return false;
-                tc_fence_after();
+            // descriptors: the 14-bit start-address field counts 16-byte units, so moving inside a tile is an
+            // addition to the low word (all tile addresses stay below the field's range: shared memory is 228 KB)
+            const unsigned long long dq = smem_desc(smem_u32(sQ), 16, 1024);                    // Q, K: K-major
+            const unsigned long long dk = smem_desc(smem_u32(ring), 16, 1024);
+            const unsigned long long dv = smem_desc(smem_u32(ring), 128 * 128, 1024);           // V: MN-major
+            auto wait_item = [&](int n) { return mbar_wait(&sh.full[n % PF_RING], (n / PF_RING) & 1, abort_flag); };
+            auto issue_S = [&](int g, int j, bool release) {      // S_g = Q_g K(j)^T; K(j) is ring item 2j
+                const int st = (2 * j) % PF_RING;
+                const unsigned long long a0 = dq + (unsigned)(g * TILE_BYTES >> 4), b0 = dk + (unsigned)(st * TILE_BYTES >> 4);
 #pragma unroll
                 for (int ks = 0; ks < D / 16; ++ks) {
-                    const unsigned off = (ks / 4) * (128 * 128) + (ks % 4) * 32;
-                    tc_mma(tmem_S[it & 1], smem_desc(q_addr + off, 16, 1024),
-                           smem_desc(k_addr + st * TILE_BYTES + off, 16, 1024), IDESC_S, ks > 0);
+                    const unsigned off = ((ks / 4) * (128 * 128) + (ks % 4) * 32) >> 4;
+                    tc_mma_ss(tmem + g * 128, a0 + off, b0 + off, IDESC_S, ks > 0);
                 }
-                tc_commit(&sh.s_full[it & 1]);
-                tc_commit(&sh.k_empty[st]);
-                return true;
+                tc_commit(&sh.s_full[g]);
+                if (release) tc_commit(&sh.empty[st]);
             };
-            int n_proc = 0;
-            for (int j = 0; j < n_tiles; ++j) n_proc += !(sh.tile[j] & (1 << 30));
-            bool ok = n_proc > 0 ? issue_S(0) : true;
-            for (int it = 0; it < n_proc && ok; ++it) {
-                if (it + 1 < n_proc) ok = issue_S(it + 1);
-                if (!ok) break;
-                const int st = it % PF_STAGES;
-                ok = mbar_wait(&sh.v_full[st], (it / PF_STAGES) & 1, abort_flag) &&
-                     mbar_wait(&sh.p_full, it & 1, abort_flag);
-                if (!ok) break;
-                tc_fence_after();
+            auto issue_PV = [&](int g, int j, bool release) {     // O_g += P_g V(j); V(j) is ring item 2j+1
+                const int st = (2 * j + 1) % PF_RING;
+                const unsigned long long b0 = dv + (unsigned)(st * TILE_BYTES >> 4);
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {   // 128 keys, 16 per MMA
-                    const unsigned a_off = (ks / 4) * (128 * 128) + (ks % 4) * 32;
-                    const unsigned b_off = st * TILE_BYTES + ks * 2048;   // 16 keys x 128 B
-                    tc_mma(tmem_O, smem_desc(p_addr + a_off, 16, 1024), smem_desc(v_addr + b_off, 128 * 128, 1024),
-                           IDESC_O, (it > 0) || (ks > 0));
+                for (int ks = 0; ks < 8; ++ks)      // 128 keys, 16 per MMA: A = 8 TMEM columns of bf16 pairs
+                    tc_mma_ts(tmem + 256 + g * 128, tmem + g * 128 + ks * 8, b0 + (unsigned)(ks * 2048 >> 4), IDESC_O,
+                              (j > 0) || (ks > 0));
+                if (release) tc_commit(&sh.empty[st]);
+            };
+            // with one issuer the thread serves both tiles in turn and releases a page after tile B's use of it
+            constexpr int NG = 3 - PF_ISSUERS;      // tiles per issuer: 1 or 2
+            bool ok = true;
+            if (n_proc > 0) {
+                ok = wait_item(0);
+                if (ok) {
+                    tc_fence_after();
+#pragma unroll
+                    for (int i = 0; i < NG; ++i) issue_S(g0 + i, 0, i == NG - 1);
                 }
-                tc_commit(&sh.pv_done);
-                tc_commit(&sh.v_empty[st]);
+            }
+            for (int j = 0; j < n_proc && ok; ++j) {
+                ok = wait_item(2 * j + 1);                                                   // V(j)
+                if (ok && j + 1 < n_proc) ok = wait_item(2 * j + 2);                         // K(j+1)
+#pragma unroll
+                for (int i = 0; i < NG && ok; ++i) {
+                    ok = mbar_wait(&sh.p_full[g0 + i], j & 1, abort_flag);                   // P(j)
+                    if (!ok) break;
+                    tc_fence_after();
+                    issue_PV(g0 + i, j, i == NG - 1);
+                    if (j + 1 < n_proc) issue_S(g0 + i, j + 1, i == NG - 1);
+                }
+            }
+            if (ok) {
+                if (n_proc > 0) tc_commit(&sh.all_done);
+                else mbar_arrive(&sh.all_done);   // nothing was issued: nothing to track
             }
         }
+        __syncwarp();
     } else {
-        // ================= softmax, correction, epilogue (one thread per row) =================
-        const int m = threadIdx.x;
-        const int mg = m0 + m;
+        // ================= softmax groups: one thread per row of tile g =================
+        const int g = warp >> 2;
+        const int m = threadIdx.x & 127;
+        const int mg = m0 + g * 128 + m;
         const int r = min(mg / G, n_q - 1);
-        const unsigned lane_base = (unsigned)(warp * 32) << 16;
+        const unsigned lane_base = (unsigned)((warp & 3) * 32) << 16;
+        const unsigned tS = tmem + g * 128 + lane_base, tO = tmem + 256 + g * 128 + lane_base;
         const float c = 1.4426950408889634f * rsqrtf((float)D);
+        const unsigned short* mrow = sh.minrow[g];
         float m_ref = -INFINITY, l = 0.f;
-        int it = 0, n_masked = 0;
+        int pi = 0, it = 0;
         bool ok = true;
         for (int j = 0; j < n_tiles && ok; ++j) {
-            const int t = sh.tile[j];
-            if (t & (1 << 30)) continue;
-            const bool masked = t & (1 << 29);
-            if (masked) {   // per-column visibility threshold for this tile
+            const unsigned t = sh.tile[j];
+            if (t >> 15) continue;
+            if (pi < p0 || pi >= p1) { ++pi; continue; }
+            ++pi;
+            const bool masked = (t >> 14) & 1;
+            unsigned vlo = 0, vlen = SVLM_PAGE;
+            if (masked) {
+                // Column m's stream ordinal relative to the first query token (clamped), shared through
+                // shared memory; it grows with the column, so the columns this row may see, valid ones with
+                // ordinal <= the row's, form the interval [lo, bound) found by bisection.
                 const SvlmTile tl = vw.tiles[j];
-                const int slot = tl.page * SVLM_PAGE + m;
-                int mr = 0x7fffffff;
+                unsigned short mr = 0xFFFF;
                 if (m >= tl.lo && m < tl.hi) {
-                    const long long rel = vw.slot_gid[slot] - gid_q0;
-                    mr = rel <= 0 ? 0 : (rel > 0x7ffffff0ll ? 0x7fffffff : (int)rel);
+                    const long long rel = vw.slot_gid[tl.page * SVLM_PAGE + m] - gid_q0;
+                    mr = rel <= 0 ? 0 : (rel > 0xFFF0ll ? 0xFFF0 : (unsigned short)rel);
                 }
-                sh.minrow[n_masked & 1][m] = mr;
-                mbar_arrive(&sh.mask_bar);                  // the 128 softmax threads meet here (bounded)
-                ok = mbar_wait(&sh.mask_bar, n_masked & 1, abort_flag);
-                if (!ok) break;
+                asm volatile("bar.sync %0, 128;" ::"r"(1 + g));   // the previous masked page's readers are done
+                sh.minrow[g][m] = mr;
+                asm volatile("bar.sync %0, 128;" ::"r"(1 + g));
+                int a = tl.lo, e = tl.hi;
+                while (a < e) {
+                    const int mid = (a + e) >> 1;
+                    if ((unsigned)mrow[mid] <= (unsigned)r) a = mid + 1; else e = mid;
+                }
+                vlo = tl.lo;
+                vlen = a - tl.lo;
             }
-            ok = mbar_wait(&sh.s_full[it & 1], (it >> 1) & 1, abort_flag);
+            ok = mbar_wait(&sh.s_full[g], it & 1, abort_flag);
             if (!ok) break;
             tc_fence_after();
-            float s[128];
-#pragma unroll
-            for (int q4 = 0; q4 < 4; ++q4) tmem_ld32(tmem_S[it & 1] + lane_base + q4 * 32, s + q4 * 32);
-            tmem_wait_ld();
-            tc_fence_before();
-            mbar_arrive(&sh.s_empty[it & 1]);
-            if (masked) {
-                const int* mr = sh.minrow[n_masked & 1];
-#pragma unroll
-                for (int k = 0; k < 128; ++k) s[k] = (r >= mr[k]) ? s[k] : -INFINITY;
-                ++n_masked;
-            }
-            float mx = s[0];
-#pragma unroll
-            for (int k = 1; k < 128; ++k) mx = fmaxf(mx, s[k]);
-            mx *= c;
-            // lazy running maximum: only move the reference when it would be exceeded by 2^8
-            const bool grow = mx > m_ref + 8.f;
-            const float m_new = grow ? mx : m_ref;
-            const float m_use = m_new == -INFINITY ? 0.f : m_new;
-            float rowsum = 0.f;
-            unsigned pk[64];
-#pragma unroll
-            for (int k = 0; k < 64; ++k) {
-                const float p0 = exp2f(fmaf(s[2 * k], c, -m_use));
-                const float p1 = exp2f(fmaf(s[2 * k + 1], c, -m_use));
-                rowsum += p0 + p1;
-                pk[k] = pack2(p0, p1);
-            }
-            // P's buffer and O are free once the previous tile's P V has completed
-            if (it > 0) {
-                ok = mbar_wait(&sh.pv_done, (it - 1) & 1, abort_flag);
-                if (!ok) break;
-                tc_fence_after();
-            }
-            const float corr = grow ? exp2f(m_ref - m_use) : 1.f;   // m_ref = -inf gives 0
-            if (it > 0 && __any_sync(0xffffffffu, grow)) {
-#pragma unroll 1
-                for (int q4 = 0; q4 < D / 32; ++q4) {
-                    float o[32];
-                    tmem_ld32(tmem_O + lane_base + q4 * 32, o);
-                    tmem_wait_ld();
-#pragma unroll
-                    for (int k = 0; k < 32; ++k) o[k] *= corr;
-                    tmem_st32(tmem_O + lane_base + q4 * 32, o);
-                }
-                tmem_wait_st();
-            }
+            float rowsum, corr, m_new;
+            if (masked) softmax_page<true>(tS, tO, D, vlo, vlen, c, m_ref, it > 0, rowsum, corr, m_new);
+            else softmax_page<false>(tS, tO, D, vlo, vlen, c, m_ref, it > 0, rowsum, corr, m_new);
+            tmem_wait_st();
             l = l * corr + rowsum;
             m_ref = m_new;
-#pragma unroll
-            for (int ch = 0; ch < 16; ++ch) {   // 16 chunks of 8 keys
-                unsigned char* dst = sP + (ch / 8) * (128 * 128) + m * 128 + (((ch % 8) ^ (m & 7)) << 4);
-                *reinterpret_cast<uint4*>(dst) = make_uint4(pk[4 * ch], pk[4 * ch + 1], pk[4 * ch + 2], pk[4 * ch + 3]);
-            }
-            fence_proxy_async();
             tc_fence_before();
-            mbar_arrive(&sh.p_full);
+            mbar_arrive(&sh.p_full[g]);
             ++it;
         }
-        // epilogue: O / l -> bf16 -> out[r][head]
-        if (ok && it > 0) ok = mbar_wait(&sh.pv_done, (it - 1) & 1, abort_flag);
-        if (ok) {
-            tc_fence_after();
-            const float inv = l > 0.f ? 1.f / l : 0.f;
+        if (ok) ok = mbar_wait(&sh.all_done, 0, abort_flag);
+        tc_fence_after();
+
+        // ---- hand-over between the two CTAs of the cluster, then the output ------------------------
+        // CTA k of the pair finishes tile k: its group 1-k sends (O, m, l) of its rows to the partner, its group k
+        // merges its own accumulator with what the partner's group k sent.  The exchange area is the K/V ring,
+        // idle once a CTA's MMAs have completed (cluster barrier #1 says so for both).
+        float* xo = reinterpret_cast<float*>(ring);                      // [D/4 chunks][128 rows] float4
+        float* xml = xo + (size_t)128 * D;                               // [128 rows][2]
+        const bool mine = n_proc > 0;                                    // this CTA processed pages
+        cluster_sync_all();   // #1: neither CTA needs its ring any more
+        if ((unsigned)g != rank) {
+            const unsigned dst_o = map_to_rank(xo, rank ^ 1), dst_ml = map_to_rank(xml, rank ^ 1);
+#pragma unroll 1
+            for (int q4 = 0; q4 < D / 32; ++q4) {
+                float o[32];
+                if (mine) { tmem_ld32(tO + q4 * 32, o); tmem_wait_ld(); }
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const float4 v = mine ? make_float4(o[4 * i], o[4 * i + 1], o[4 * i + 2], o[4 * i + 3])
+                                          : make_float4(0.f, 0.f, 0.f, 0.f);
+                    st_cluster_v4(dst_o + (unsigned)(((q4 * 8 + i) * 128 + m) * 16), v);
+                }
+            }
+            st_cluster_v2(dst_ml + (unsigned)(m * 8), make_float2(ok && mine ? m_ref : -INFINITY, ok && mine ? l : 0.f));
+        }
+        cluster_sync_all();   // #2: the partner's rows have arrived
+        if ((unsigned)g == rank && ok) {
+            const float mb = xml[m * 2], lb = xml[m * 2 + 1];
+            const float ma = mine ? m_ref : -INFINITY, la = mine ? l : 0.f;
+            const float M = fmaxf(ma, mb);
+            const float fa = ma == -INFINITY ? 0.f : exp2f(ma - M), fb = mb == -INFINITY ? 0.f : exp2f(mb - M);
+            const float L = la * fa + lb * fb;
+            const float inv = L > 0.f ? 1.f / L : 0.f;
+            const float ga = fa * inv, gb = fb * inv;
             const bool live = mg < m_total;
             uint16_t* dst = out + ((((size_t)prob) * n_q + r) * q_heads + hk * G + (mg % G)) * D;
 #pragma unroll 1
             for (int q4 = 0; q4 < D / 32; ++q4) {
                 float o[32];
-                if (it > 0) {
-                    tmem_ld32(tmem_O + lane_base + q4 * 32, o);
-                    tmem_wait_ld();
-                } else {
+                if (mine) { tmem_ld32(tO + q4 * 32, o); tmem_wait_ld(); }
 #pragma unroll
-                    for (int k = 0; k < 32; ++k) o[k] = 0.f;
+                for (int i = 0; i < 8; ++i) {
+                    const float4 pb = *reinterpret_cast<const float4*>(xo + (size_t)((q4 * 8 + i) * 128 + m) * 4);
+                    o[4 * i] = (ma > -INFINITY ? o[4 * i] * ga : 0.f) + (mb > -INFINITY ? pb.x * gb : 0.f);
+                    o[4 * i + 1] = (ma > -INFINITY ? o[4 * i + 1] * ga : 0.f) + (mb > -INFINITY ? pb.y * gb : 0.f);
+                    o[4 * i + 2] = (ma > -INFINITY ? o[4 * i + 2] * ga : 0.f) + (mb > -INFINITY ? pb.z * gb : 0.f);
+                    o[4 * i + 3] = (ma > -INFINITY ? o[4 * i + 3] * ga : 0.f) + (mb > -INFINITY ? pb.w * gb : 0.f);
                 }
                 if (live) {
 #pragma unroll
                     for (int k = 0; k < 4; ++k) {
                         uint4 v;
-                        v.x = pack2(o[8 * k] * inv, o[8 * k + 1] * inv);
-                        v.y = pack2(o[8 * k + 2] * inv, o[8 * k + 3] * inv);
-                        v.z = pack2(o[8 * k + 4] * inv, o[8 * k + 5] * inv);
-                        v.w = pack2(o[8 * k + 6] * inv, o[8 * k + 7] * inv);
+                        v.x = pack2(o[8 * k], o[8 * k + 1]);
+                        v.y = pack2(o[8 * k + 2], o[8 * k + 3]);
+                        v.z = pack2(o[8 * k + 4], o[8 * k + 5]);
+                        v.w = pack2(o[8 * k + 6], o[8 * k + 7]);
                         *reinterpret_cast<uint4*>(dst + q4 * 32 + 8 * k) = v;
                     }
                 }
             }
         }
+    }
+    if (warp >= 8) {          // the producer and issuer warps take part in the two cluster barriers as well
+        cluster_sync_all();
+        cluster_sync_all();
     }
 
     // ---- teardown ------------------------------------------------------------------------------
@@ -436,23 +581,48 @@ prefill_kernel(SvlmAttendBatch b, int layer0, int n_layers, const uint16_t* __re
         // Somebody gave up.  Copies already issued still land in this CTA's shared memory: give
         // every full-barrier a bounded chance to complete before the memory is released.
         if (threadIdx.x == 0) {
-            for (int s = 0; s < PF_STAGES; ++s)
-                for (unsigned p = 0; p < 2; ++p) {
-                    for (unsigned w = 0; w < (1u << 16) && !mbar_test(&sh.k_full[s], p); ++w) __nanosleep(32);
-                    for (unsigned w = 0; w < (1u << 16) && !mbar_test(&sh.v_full[s], p); ++w) __nanosleep(32);
-                }
+            for (int s = 0; s < PF_RING; ++s)
+                for (unsigned p = 0; p < 2; ++p)
+                    for (unsigned w = 0; w < (1u << 16) && !mbar_test(&sh.full[s], p); ++w) __nanosleep(32);
             atomicCAS(const_cast<int*>(&vw.ctrl->status), 0, -5);   // SVLM_ERR_TIMEOUT
         }
         __syncthreads();
     }
-    if (warp == 4) {
+    if (warp == 8) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512));
     }
 }
 
 template <int D>
-constexpr size_t prefill_smem() { return sizeof(PfShared) + 1024 + (size_t)(1 + 2 * PF_STAGES + 1) * 128 * D * 2 + (D == 64 ? 128 * 128 : 0); }
+constexpr size_t prefill_smem() { return sizeof(PfShared) + 1024 + (size_t)(2 + PF_RING) * 128 * D * 2; }
+
+template <int D>
+cudaError_t launch(const SvlmAttendBatch& b, int layer0, int n_layers, const uint16_t* Q, const int* q_pos, int n_q,
+                   int q_heads, uint16_t* out, cudaStream_t st) {
+    static bool once = false;
+    cudaError_t e;
+    if (!once) {
+        e = cudaFuncSetAttribute(prefill_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)prefill_smem<D>());
+        if (e != cudaSuccess) return e;
+        once = true;
+    }
+    const int G = q_heads / b.kv_heads;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * ((n_q * G + PF_ROWS - 1) / PF_ROWS), b.kv_heads, b.n_caches * n_layers);
+    cfg.blockDim = dim3(PF_THREADS);
+    cfg.dynamicSmemBytes = prefill_smem<D>();
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;     // the two CTAs that share the pages of one row tile
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    e = cudaLaunchKernelEx(&cfg, prefill_kernel<D>, b, layer0, n_layers, Q, q_pos, n_q, q_heads, out);
+    return e != cudaSuccess ? e : cudaGetLastError();
+}
 
 }  // namespace
 
@@ -460,28 +630,9 @@ bool svlm_prefill_supported(int n_pages, int group) { return n_pages <= PF_MAX_T
 
 cudaError_t svlm_launch_prefill(const SvlmAttendBatch& b, int layer0, int n_layers, const void* Q, const int* q_pos,
                                 int n_q, int q_heads, void* out, cudaStream_t st) {
-    const int G = q_heads / b.kv_heads;
-    dim3 grid((n_q * G + 127) / 128, b.kv_heads, b.n_caches * n_layers);
-    cudaError_t e;
-    if (b.head_dim == 128) {
-        static bool once = false;
-        if (!once) {
-            e = cudaFuncSetAttribute(prefill_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)prefill_smem<128>());
-            if (e != cudaSuccess) return e;
-            once = true;
-        }
-        prefill_kernel<128><<<grid, PF_THREADS, prefill_smem<128>(), st>>>(b, layer0, n_layers, (const uint16_t*)Q, q_pos,
-                                                                        n_q, q_heads, (uint16_t*)out);
-    } else {
-        static bool once = false;
-        if (!once) {
-            e = cudaFuncSetAttribute(prefill_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)prefill_smem<64>());
-            if (e != cudaSuccess) return e;
-            once = true;
-        }
-        prefill_kernel<64><<<grid, PF_THREADS, prefill_smem<64>(), st>>>(b, layer0, n_layers, (const uint16_t*)Q, q_pos,
-                                                                      n_q, q_heads, (uint16_t*)out);
-    }
+    const cudaError_t e = b.head_dim == 128
+        ? launch<128>(b, layer0, n_layers, (const uint16_t*)Q, q_pos, n_q, q_heads, (uint16_t*)out, st)
+        : launch<64>(b, layer0, n_layers, (const uint16_t*)Q, q_pos, n_q, q_heads, (uint16_t*)out, st);
     svlm_count_launch();
-    return cudaGetLastError();
+    return e;
 }
