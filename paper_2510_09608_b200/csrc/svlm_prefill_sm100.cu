@@ -96,6 +96,13 @@ __device__ __forceinline__ void tmem_st16(unsigned taddr, const unsigned* r) {
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
+// One lane of the (converged) warp.
+__device__ __forceinline__ bool elect_one() {
+    unsigned pred;
+    asm volatile("{\n.reg .pred p;\nelect.sync _|p, 0xffffffff;\nselp.u32 %0, 1, 0, p;\n}" : "=r"(pred));
+    return pred != 0;
+}
+
 // Hardware barrier of the thread-block cluster (every thread of both CTAs takes part).
 __device__ __forceinline__ void cluster_sync_all() {
     asm volatile("barrier.cluster.arrive.release.aligned;\nbarrier.cluster.wait.acquire.aligned;" ::: "memory");
@@ -321,11 +328,25 @@ prefill_kernel(SvlmAttendBatch b, int layer0, int n_layers, const uint16_t* __re
     const int n_tok = r_hi - r_lo + 1;
     const bool cs_shared = (size_t)n_tok * HALF * sizeof(float2) <= (size_t)2 * TILE_BYTES;
     if (cs_shared) {
-        for (int i = threadIdx.x; i < n_tok * HALF; i += PF_THREADS) {
-            const int tk = i / HALF, pair = i % HALF;
-            const int axis = b.rope_mode == 0 ? 0 : (pair < b.sec_t ? 0 : (pair < b.sec_th ? 1 : 2));
-            const int* qp = q_pos + ((size_t)ci * n_q + r_lo + tk) * (b.rope_mode == 0 ? 1 : 3);
-            s_cs[i] = svlm_rope_cs(tab, HALF, pair, (long long)qp[b.rope_mode == 0 ? 0 : axis] - shift, b.theta[pair]);
+        constexpr int UN = 8;   // entries per thread in flight: positions first, then the table look-ups
+        const int n_ent = n_tok * HALF;
+        const int pw = b.rope_mode == 0 ? 1 : 3;
+        for (int base = 0; base < n_ent; base += PF_THREADS * UN) {
+            long long cpos[UN];
+#pragma unroll
+            for (int u = 0; u < UN; ++u) {
+                const int i = base + u * PF_THREADS + threadIdx.x;
+                if (i < n_ent) {
+                    const int tk = i / HALF, pair = i % HALF;
+                    const int axis = b.rope_mode == 0 ? 0 : (pair < b.sec_t ? 0 : (pair < b.sec_th ? 1 : 2));
+                    cpos[u] = (long long)__ldg(q_pos + ((size_t)ci * n_q + r_lo + tk) * pw + axis) - shift;
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < UN; ++u) {
+                const int i = base + u * PF_THREADS + threadIdx.x;
+                if (i < n_ent) s_cs[i] = svlm_rope_cs(tab, HALF, i % HALF, cpos[u], b.theta[i % HALF]);
+            }
         }
     }
     __syncthreads();
@@ -339,14 +360,30 @@ prefill_kernel(SvlmAttendBatch b, int layer0, int n_layers, const uint16_t* __re
         const float2* cs_row = s_cs + (size_t)(r - r_lo) * HALF;
         const int* qp = q_pos + ((size_t)ci * n_q + r) * (b.rope_mode == 0 ? 1 : 3);
         unsigned char* sQg = sQ + g * TILE_BYTES;
-        uint4 rowv[D / 8];                         // the whole row: every load in flight before the first use
-#pragma unroll
-        for (int i = 0; i < D / 8; ++i) rowv[i] = live ? __ldg(reinterpret_cast<const uint4*>(src) + i) : make_uint4(0, 0, 0, 0);
-#pragma unroll
+        // (a compact loop: the code runs once per thread, so its instruction footprint matters more than its
+        //  schedule; the next chunk's loads are issued before the current chunk is rotated)
+        auto ld_chunk = [&](int i) { return live ? __ldg(reinterpret_cast<const uint4*>(src) + i) : make_uint4(0, 0, 0, 0); };
+        uint4 lo_n = ld_chunk(0), hi_n = ld_chunk(HALF / 8);
+#pragma unroll 1
         for (int c8 = 0; c8 < HALF / 8; ++c8) {    // 8 pairs at a time: chunk c8 of the low half, same of the high half
-            const uint4 lo4 = rowv[c8], hi4 = rowv[HALF / 8 + c8];
+            const uint4 lo4 = lo_n, hi4 = hi_n;
+            if (c8 + 1 < HALF / 8) { lo_n = ld_chunk(c8 + 1); hi_n = ld_chunk(HALF / 8 + c8 + 1); }
             const unsigned* lw = reinterpret_cast<const unsigned*>(&lo4);
             const unsigned* hw = reinterpret_cast<const unsigned*>(&hi4);
+            float2 cs8[8];
+            if (cs_shared) {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) cs8[i] = cs_row[c8 * 8 + i];
+            } else {
+#pragma unroll 1
+                for (int i = 0; i < 8; ++i) {      // direct look-ups (too many tokens for the shared table)
+                    const int pair = c8 * 8 + i;
+                    const int axis = b.rope_mode == 0 ? 0 : (pair < b.sec_t ? 0 : (pair < b.sec_th ? 1 : 2));
+                    const float2 v = svlm_rope_cs(tab, HALF, pair, (long long)qp[b.rope_mode == 0 ? 0 : axis] - shift, b.theta[pair]);
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) if (q == i) cs8[q] = v;
+                }
+            }
             unsigned lo_o[4], hi_o[4];
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
@@ -355,14 +392,7 @@ prefill_kernel(SvlmAttendBatch b, int layer0, int n_layers, const uint16_t* __re
                 float ol[2], oh[2];
 #pragma unroll
                 for (int e = 0; e < 2; ++e) {
-                    const int pair = c8 * 8 + 2 * j + e;
-                    float2 cs;
-                    if (cs_shared) {
-                        cs = cs_row[pair];
-                    } else {
-                        const int axis = b.rope_mode == 0 ? 0 : (pair < b.sec_t ? 0 : (pair < b.sec_th ? 1 : 2));
-                        cs = svlm_rope_cs(tab, HALF, pair, (long long)qp[b.rope_mode == 0 ? 0 : axis] - shift, b.theta[pair]);
-                    }
+                    const float2 cs = cs8[2 * j + e];
                     ol[e] = xl[e] * cs.x - xh[e] * cs.y;
                     oh[e] = xh[e] * cs.x + xl[e] * cs.y;
                 }
@@ -393,8 +423,12 @@ prefill_kernel(SvlmAttendBatch b, int layer0, int n_layers, const uint16_t* __re
         // Per tile the order is S(0) | PV(j) S(j+1) | ...: the tensor pipe executes one thread's instructions in
         // order, so S(j+1) overwrites the columns of P(j) only after PV(j) has read them.  Two issuing threads keep
         // the pipe fed while one of them sits in a wait.
-        if (lane == 0 && warp - 9 < PF_ISSUERS) {
+        // The whole warp runs the loop (waits, descriptor arithmetic: warp-uniform values the compiler can keep in
+        // uniform registers); one elected lane executes the tcgen05 instructions.
+        if (warp - 9 < PF_ISSUERS) {
             const int g0 = warp - 9;
+            const unsigned tmem = __shfl_sync(0xffffffffu, sh.tmem_base, 0);
+            const bool leader = elect_one();
             constexpr unsigned IDESC_S = make_idesc(128, 128, 0);
             constexpr unsigned IDESC_O = make_idesc(128, D, 1);
             // descriptors: the 14-bit start-address field counts 16-byte units, so moving inside a tile is an
@@ -402,26 +436,38 @@ prefill_kernel(SvlmAttendBatch b, int layer0, int n_layers, const uint16_t* __re
             const unsigned long long dq = smem_desc(smem_u32(sQ), 16, 1024);                    // Q, K: K-major
             const unsigned long long dk = smem_desc(smem_u32(ring), 16, 1024);
             const unsigned long long dv = smem_desc(smem_u32(ring), 128 * 128, 1024);           // V: MN-major
-            auto wait_item = [&](int n) { return mbar_wait(&sh.full[n % PF_RING], (n / PF_RING) & 1, abort_flag); };
+            // every wait gives the same answer in all lanes, so the warp stays converged
+            auto wait_bar = [&](void* bar, unsigned parity) {   // one lane polls, all lanes get the answer
+                int r = 1;
+                if (lane == 0) r = mbar_wait(bar, parity, abort_flag);
+                return __shfl_sync(0xffffffffu, r, 0) != 0;
+            };
+            auto wait_item = [&](int n) { return wait_bar(&sh.full[n % PF_RING], (n / PF_RING) & 1); };
             auto issue_S = [&](int g, int j, bool release) {      // S_g = Q_g K(j)^T; K(j) is ring item 2j
                 const int st = (2 * j) % PF_RING;
                 const unsigned long long a0 = dq + (unsigned)(g * TILE_BYTES >> 4), b0 = dk + (unsigned)(st * TILE_BYTES >> 4);
+                if (leader) {
 #pragma unroll
-                for (int ks = 0; ks < D / 16; ++ks) {
-                    const unsigned off = ((ks / 4) * (128 * 128) + (ks % 4) * 32) >> 4;
-                    tc_mma_ss(tmem + g * 128, a0 + off, b0 + off, IDESC_S, ks > 0);
+                    for (int ks = 0; ks < D / 16; ++ks) {
+                        const unsigned off = ((ks / 4) * (128 * 128) + (ks % 4) * 32) >> 4;
+                        tc_mma_ss(tmem + g * 128, a0 + off, b0 + off, IDESC_S, ks > 0);
+                    }
+                    tc_commit(&sh.s_full[g]);
+                    if (release) tc_commit(&sh.empty[st]);
                 }
-                tc_commit(&sh.s_full[g]);
-                if (release) tc_commit(&sh.empty[st]);
+                __syncwarp();
             };
             auto issue_PV = [&](int g, int j, bool release) {     // O_g += P_g V(j); V(j) is ring item 2j+1
                 const int st = (2 * j + 1) % PF_RING;
                 const unsigned long long b0 = dv + (unsigned)(st * TILE_BYTES >> 4);
+                if (leader) {
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks)      // 128 keys, 16 per MMA: A = 8 TMEM columns of bf16 pairs
-                    tc_mma_ts(tmem + 256 + g * 128, tmem + g * 128 + ks * 8, b0 + (unsigned)(ks * 2048 >> 4), IDESC_O,
-                              (j > 0) || (ks > 0));
-                if (release) tc_commit(&sh.empty[st]);
+                    for (int ks = 0; ks < 8; ++ks)      // 128 keys, 16 per MMA: A = 8 TMEM columns of bf16 pairs
+                        tc_mma_ts(tmem + 256 + g * 128, tmem + g * 128 + ks * 8, b0 + (unsigned)(ks * 2048 >> 4), IDESC_O,
+                                  (j > 0) || (ks > 0));
+                    if (release) tc_commit(&sh.empty[st]);
+                }
+                __syncwarp();
             };
             // with one issuer the thread serves both tiles in turn and releases a page after tile B's use of it
             constexpr int NG = 3 - PF_ISSUERS;      // tiles per issuer: 1 or 2
@@ -439,14 +485,14 @@ prefill_kernel(SvlmAttendBatch b, int layer0, int n_layers, const uint16_t* __re
                 if (ok && j + 1 < n_proc) ok = wait_item(2 * j + 2);                         // K(j+1)
 #pragma unroll
                 for (int i = 0; i < NG && ok; ++i) {
-                    ok = mbar_wait(&sh.p_full[g0 + i], j & 1, abort_flag);                   // P(j)
+                    ok = wait_bar(&sh.p_full[g0 + i], j & 1);                                 // P(j)
                     if (!ok) break;
                     tc_fence_after();
                     issue_PV(g0 + i, j, i == NG - 1);
                     if (j + 1 < n_proc) issue_S(g0 + i, j + 1, i == NG - 1);
                 }
             }
-            if (ok) {
+            if (ok && leader) {
                 if (n_proc > 0) tc_commit(&sh.all_done);
                 else mbar_arrive(&sh.all_done);   // nothing was issued: nothing to track
             }
