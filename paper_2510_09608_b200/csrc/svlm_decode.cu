@@ -9,7 +9,7 @@
 //   * one producer thread streams the sub-tiles with TMA (2D boxes of 32 keys x 64 dims, 128-byte
 //     swizzle) through a ring of shared-memory stages, each with a full and an empty mbarrier;
 //     the whole first ring-load is in flight before anything else happens;
-//   * four consumer warps take sub-tiles round-robin; the G <= 8 query heads that share a KV head
+//   * six consumer warps take sub-tiles round-robin, each through its own ring stage; the G <= 8 query heads that share a KV head
 //     ride in the N dimension of m16n8k16 MMAs (S^T = K Q^T, O^T += V^T P^T), so K and V are read
 //     once for the whole group; per-warp online softmax with warp-shuffle reductions;
 //   * rotation factors come from a small table (no sincos in the kernel);
@@ -35,9 +35,12 @@ namespace {
 
 using namespace svlm_ptx;
 
-constexpr int DEC_CWARPS = 8;                       // consumer warps
+constexpr int DEC_CWARPS = 6;                       // consumer warps
 constexpr int DEC_THREADS = (DEC_CWARPS + 1) * 32;  // + one producer warp
-constexpr int DEC_STAGES = 6;
+// One ring stage per consumer warp: a warp meets every phase of its stage's barriers in turn.  (With
+// a stage shared between warps a waiter would skip phases, and a parity wait cannot tell the phase
+// it wants from the one two earlier.)
+constexpr int DEC_STAGES = DEC_CWARPS;
 constexpr int SUB = 32;                             // keys per sub-tile
 constexpr int DEC_MAX_TILES = 512;
 
@@ -436,7 +439,8 @@ decode_kernel(SvlmAttendBatch b, int layer0, int n_layers, const uint16_t* __res
     const unsigned char* parts = ws_parts + (size_t)(li * b.kv_heads + hk) * splits * REC;
     constexpr int PER_ROUND = DEC_STAGES * STAGE_BYTES / REC;
     const int pairs = G * (D / 8);                      // groups of eight output elements
-    const int grp = threadIdx.x >> 1, sub = threadIdx.x & 1;
+    const bool two = pairs * 2 <= DEC_THREADS;          // otherwise one thread takes all records of its group
+    const int grp = two ? threadIdx.x >> 1 : threadIdx.x, sub = two ? threadIdx.x & 1 : 0, stride = two ? 2 : 1;
     const bool owner = grp < pairs;
     const int h = grp / (D / 8), d0 = (grp % (D / 8)) * 8;
     float M = -INFINITY, L = 0.f;
@@ -465,7 +469,7 @@ decode_kernel(SvlmAttendBatch b, int layer0, int n_layers, const uint16_t* __res
 #pragma unroll
                 for (int e = 0; e < 8; ++e) acc[e] *= resc;
 #pragma unroll 4
-                for (int r = sub; r < n; r += 2) {
+                for (int r = sub; r < n; r += stride) {
                     const unsigned char* rec = ring + (size_t)r * REC;
                     const float w = exp2f(*reinterpret_cast<const float*>(rec + 8 * D * 2 + h * 4) - Mn);
                     L += *reinterpret_cast<const float*>(rec + 8 * D * 2 + 32 + h * 4) * w;
@@ -480,9 +484,11 @@ decode_kernel(SvlmAttendBatch b, int layer0, int n_layers, const uint16_t* __res
         }
     }
     // even + odd records (both threads of a pair used the same maximum)
-    L += __shfl_xor_sync(0xffffffffu, L, 1);
+    if (two) {
+        L += __shfl_xor_sync(0xffffffffu, L, 1);
 #pragma unroll
-    for (int e = 0; e < 8; ++e) acc[e] += __shfl_xor_sync(0xffffffffu, acc[e], 1);
+        for (int e = 0; e < 8; ++e) acc[e] += __shfl_xor_sync(0xffffffffu, acc[e], 1);
+    }
     if (owner && sub == 0) {
         const float inv = L > 0.f ? 1.f / L : 0.f;
         uint4 pk;

@@ -364,7 +364,7 @@ prefill_kernel(SvlmAttendBatch b, int layer0, int n_layers, const uint16_t* __re
         //  schedule; the next chunk's loads are issued before the current chunk is rotated)
         auto ld_chunk = [&](int i) { return live ? __ldg(reinterpret_cast<const uint4*>(src) + i) : make_uint4(0, 0, 0, 0); };
         uint4 lo_n = ld_chunk(0), hi_n = ld_chunk(HALF / 8);
-#pragma unroll 1
+#pragma unroll 2
         for (int c8 = 0; c8 < HALF / 8; ++c8) {    // 8 pairs at a time: chunk c8 of the low half, same of the high half
             const uint4 lo4 = lo_n, hi4 = hi_n;
             if (c8 + 1 < HALF / 8) { lo_n = ld_chunk(c8 + 1); hi_n = ld_chunk(HALF / 8 + c8 + 1); }

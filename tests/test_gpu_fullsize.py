@@ -1,0 +1,210 @@
+"""GPU parity at the full workload sizes, in the launch configuration the benchmark times.
+
+The streams are too long to compare every value, so the CPU checker follows the *metadata* of every
+token (cheap) and receives keys/values only for the layers that are compared; every input value is
+regenerable from its coordinates.  Compared: kept ordinals, positions and total shift bit-exactly;
+stored keys of sampled layers within the re-rotation rounding bound, values bit-exactly; attention
+outputs of sampled query rows (the first, the last and a seeded random set) of sampled layers for the
+chunk prefill, and every decode output of those layers, within the acceptance band.
+"""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+pytestmark = pytest.mark.gpu
+
+
+def _setup(wl, stream_id=0):
+    import oracle
+    from paper_2510_09608_b200 import binding, streamgen as sg
+    stream = sg.Stream(wl, stream_id)
+    cache = binding.Cache(wl.layers, wl.kv_heads, wl.head_dim, wl.n_sink, wl.vision_window, wl.text_window, wl.capacity)
+    cache.set_rope(wl.rope_mode, wl.rope_base, wl.sections)
+    ref = oracle.Oracle(wl.layers, wl.kv_heads, wl.head_dim, wl.n_sink, wl.vision_window, wl.text_window,
+                        rope_mode=wl.rope_mode, rope_base=wl.rope_base, sections=wl.sections)
+    return stream, cache, ref
+
+
+def _fill(cache, ref, wl, stream):
+    """Stream chunks (append + evict, decode tokens appended in bulk) through both sides until every window is
+    full; the checker only follows the metadata."""
+    from paper_2510_09608_b200 import streamgen as sg
+    gen = lambda tensor, g: torch.stack(  # noqa: E731
+        [sg.rows_bf16_torch(wl.seed, tensor, stream.stream, l, g, wl.kv_heads, wl.head_dim) for l in range(wl.layers)])
+    n_text, chunks, evicts = 0, 0, 0
+    while n_text < wl.n_sink + wl.text_window + 64 or chunks * wl.vision_per_chunk < wl.vision_window + 1:
+        gids, types, pos = stream.next_chunk()
+        extra = [stream.next_decode_token() for _ in range(wl.decode_steps)]
+        cache.append(-1, gen(sg.TENSOR_K, gids), gen(sg.TENSOR_V, gids), torch.from_numpy(types).cuda(),
+                     torch.from_numpy(np.ascontiguousarray(pos)).cuda())
+        cache.evict()
+        ref.append(None, None, types, pos)
+        ref.evict()
+        evicts += 1
+        if extra:
+            g = np.concatenate([e[0] for e in extra]); t = np.concatenate([e[1] for e in extra])
+            p = np.concatenate([e[2] for e in extra])
+            cache.append(-1, gen(sg.TENSOR_K, g), gen(sg.TENSOR_V, g), torch.from_numpy(t).cuda(),
+                         torch.from_numpy(np.ascontiguousarray(p)).cuda())
+            ref.append(None, None, t, p)
+        n_text += int((types == sg.TEXT).sum()) + len(extra)
+        chunks += 1
+    return evicts
+
+
+def _same_metadata(cache, ref):
+    from paper_2510_09608_b200 import binding
+    got, want = cache.query(), ref.query()
+    assert cache.status() == binding.OK
+    assert np.array_equal(got["gids"], want["gids"]), "kept set differs"
+    assert np.array_equal(got["types"], want["types"])
+    assert np.array_equal(got["pos"], want["pos"]), "positions differ"
+    assert got["shift_total"] == want["shift_total"]
+
+
+def _give(ref, stream, layer):
+    gids = ref.query()["gids"]
+    ref.set_kv(layer, gids, stream.k(layer, gids), stream.v(layer, gids))
+
+
+def _give_new(ref, stream, layer, gids):
+    """Values of freshly appended tokens only (the kept history already has them)."""
+    ref.set_kv(layer, gids, stream.k(layer, gids), stream.v(layer, gids))
+
+
+def _check_kv(cache, ref, stream, wl, layer, n_evicts):
+    from paper_2510_09608_b200 import streamgen as sg
+    _give(ref, stream, layer)
+    Kb, Vb = cache.read_kv(layer, ref.count())
+    want_k, want_v = ref.rotated_k(layer), ref.values(layer)
+    assert np.array_equal(sg.bf16_bits_to_f64(Vb), want_v), "values must be bit-exact"
+    half = wl.head_dim // 2
+    pn = np.sqrt(want_k[..., :half] ** 2 + want_k[..., half:] ** 2)
+    pn = np.concatenate([pn, pn], axis=-1)
+    # every (re-)rotation rounds to bf16 once: |err| <= 2^-8 * pair norm per rounding
+    err = np.abs(sg.bf16_bits_to_f64(Kb) - want_k)
+    assert np.all(err <= (n_evicts + 1) * 2.0 ** -8 * 1.05 * pn + 1e-6), f"key error {err.max()} exceeds the rounding bound"
+
+
+def _close(got, want, what):
+    from harness import MAX_ABS, MEAN_ABS
+    err = np.abs(got - want)
+    assert err.max() <= MAX_ABS and err.mean() <= MEAN_ABS, f"{what}: max {err.max()}, mean {err.mean()}"
+    rms = np.sqrt((err ** 2).mean()) / max(np.sqrt((want ** 2).mean()), 1e-30)
+    assert rms <= 0.03, f"{what}: rms error is {rms:.4f} of the rms signal"
+
+
+def test_config3_full_stack_steady_state_step_as_benchmarked():
+    """28 layers at the deployed policy (512 sinks / 8192 vision / 512 text), steady state, two steps run exactly
+    as bench.py runs them: layer-sequential C-ABI calls replayed from a CUDA graph (append + evict + per-layer
+    append/prefill + 16 fused decode steps per layer)."""
+    import bench
+    from harness import dev_to_f64
+    from paper_2510_09608_b200 import streamgen as sg
+    wl = sg.workloads()[3]
+    stream, cache, ref = _setup(wl)
+    n_evicts = _fill(cache, ref, wl, stream)
+    _same_metadata(cache, ref)
+    layers = (0, 13, 27)
+    rng = np.random.default_rng(wl.seed)
+    for step in range(2):
+        chunk, decode = bench.next_step_schedule(stream, wl)
+        inp = bench.StepInputs(wl, stream, chunk, decode)
+        if step == 0:      # one plain step on a scratch cache sets the kernels' one-time attributes outside the capture
+            _, scratch, _ = _setup(wl)
+            bench.run_step(scratch, wl, inp)
+            torch.cuda.synchronize()
+            scratch.close()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            cache.set_stream(torch.cuda.current_stream())
+            bench.run_step(cache, wl, inp)
+        cache.set_stream(torch.cuda.current_stream())
+        g.replay()
+        torch.cuda.synchronize()
+        # the checker walks the same step and produces the expected values at each point
+        gids, types, pos = chunk
+        ref.append(None, None, types, pos)
+        ref.evict()
+        n_evicts += 1
+        rows = np.unique(np.concatenate([[0, len(gids) - 1], rng.integers(0, len(gids), 16)]))
+        for l in layers:
+            _give(ref, stream, l)
+            want = ref.attend(l, stream.q(l, gids), pos, rows)
+            _close(dev_to_f64(inp.out[l])[rows], want, f"step {step} prefill layer {l}")
+        for d, (g1, t1, p1) in zip(inp.dec, decode):
+            ref.append(None, None, t1, p1)
+            for l in layers:
+                _give_new(ref, stream, l, g1)
+                _close(dev_to_f64(d["out"][l]), ref.attend(l, stream.q(l, g1), p1), f"step {step} decode layer {l}")
+        _same_metadata(cache, ref)
+    for l in layers:
+        _check_kv(cache, ref, stream, wl, l, n_evicts)
+
+
+def test_config4_batched_decode_16_streams_with_interleaved_eviction():
+    """16 independent streams at the full retained size, 48 batched q=1 steps (one launch for all streams), an
+    eviction every 16 steps; every stream's output compared at sampled steps, metadata after every eviction."""
+    from harness import bits_to_dev, dev_to_f64
+    from paper_2510_09608_b200 import binding, streamgen as sg
+    wl = dataclasses.replace(sg.workloads()[4], decode_steps=16)
+    sides = []
+    for sid in range(wl.streams):
+        stream, cache, ref = _setup(wl, sid)
+        _fill(cache, ref, wl, stream)
+        _give(ref, stream, 0)
+        sides.append((stream, cache, ref))
+    for step in range(48):
+        toks = [s.next_decode_token() for s, _, _ in sides]
+        for (s, c, r), (g1, t1, p1) in zip(sides, toks):
+            c.append(0, bits_to_dev(s.k(0, g1)), bits_to_dev(s.v(0, g1)), torch.from_numpy(t1).cuda(),
+                     torch.from_numpy(np.ascontiguousarray(p1)).cuda())
+            r.append(None, None, t1, p1)
+            _give_new(r, s, 0, g1)
+        Q = np.stack([s.q(0, g1) for (s, _, _), (g1, _, _) in zip(sides, toks)])
+        qpos = torch.from_numpy(np.stack([p1 for _, _, p1 in toks])).cuda()
+        out = dev_to_f64(binding.attend_batched([c for _, c, _ in sides], 0, bits_to_dev(Q), qpos))
+        if step % 16 in (0, 15):
+            for i, ((s, c, r), (g1, t1, p1)) in enumerate(zip(sides, toks)):
+                _close(out[i], r.attend(0, Q[i], p1), f"stream {i} step {step}")
+        if step % 16 == 15:
+            for s, c, r in sides:
+                c.evict()
+                r.evict()
+                _same_metadata(c, r)
+
+
+def test_config5_high_frame_rate_streams_sampled():
+    """The 8 frames/s x 8x8-grid shape (vision blocks of span 8, text bursts up to 32): two of the eight streams,
+    four of the 28 layers, one steady-state step each, layer-sequential calls as benchmarked."""
+    import bench
+    from harness import dev_to_f64
+    from paper_2510_09608_b200 import streamgen as sg
+    wl = dataclasses.replace(sg.workloads()[5], layers=4)
+    rng = np.random.default_rng(wl.seed)
+    for sid in (0, 7):
+        stream, cache, ref = _setup(wl, sid)
+        n_evicts = _fill(cache, ref, wl, stream)
+        _same_metadata(cache, ref)
+        chunk, decode = bench.next_step_schedule(stream, wl)
+        inp = bench.StepInputs(wl, stream, chunk, decode)
+        bench.run_step(cache, wl, inp)
+        torch.cuda.synchronize()
+        gids, types, pos = chunk
+        ref.append(None, None, types, pos)
+        ref.evict()
+        rows = np.unique(np.concatenate([[0, len(gids) - 1], rng.integers(0, len(gids), 16)]))
+        for l in (0, 3):
+            _give(ref, stream, l)
+            _close(dev_to_f64(inp.out[l])[rows], ref.attend(l, stream.q(l, gids), pos, rows), f"stream {sid} prefill layer {l}")
+        for d, (g1, t1, p1) in zip(inp.dec, decode):
+            ref.append(None, None, t1, p1)
+            for l in (0, 3):
+                _give_new(ref, stream, l, g1)
+        for l in (0, 3):
+            g1, t1, p1 = decode[-1]
+            _close(dev_to_f64(inp.dec[-1]["out"][l]), ref.attend(l, stream.q(l, g1), p1), f"stream {sid} last decode layer {l}")
+        _same_metadata(cache, ref)
+        _check_kv(cache, ref, stream, wl, 3, n_evicts + 1)

@@ -109,6 +109,25 @@ def test_degenerate_policies(S, Vw, Tw):
         assert_close(s.attend(0))
 
 
+def test_eight_query_heads_per_kv_head_and_all_layers_decode():
+    """The widest group the tensor-core decode kernel packs (8 query heads per KV head), through single-layer,
+    fused and all-layers (one launch, one CTA streaming many sub-tiles) decode calls."""
+    from harness import SideBySide, assert_close
+    wl = dataclasses.replace(_wl(2), layers=3, q_heads=16, kv_heads=2, n_sink=24, vision_window=5 * 128, text_window=90,
+                             frames=2, grid_h=8, grid_w=8, text_max=24, decode_steps=3)
+    s = SideBySide(wl)
+    for chunk in range(9):
+        s.append_chunk()
+        s.evict()
+        s.check_metadata()
+        assert_close(s.attend(chunk % 3))
+        for st in s.decode_step_fused():
+            assert_close(st)
+        s.append_decode_token()
+        assert_close(s.attend(1))
+        assert_close(s.attend(2, all_layers=True))
+
+
 def test_batched_streams_match_single_calls():
     from harness import SideBySide, bits_to_dev, dev_to_f64
     from paper_2510_09608_b200 import binding
