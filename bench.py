@@ -201,6 +201,17 @@ def fill_to_steady_state(cache, wl, stream):
     return chunks
 
 
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the attention and eviction kernels from the
+# ncu captures summarised under profiles/ (*_kernel_config3_8layers.txt; one layer per attention launch, so the
+# per-launch traffic is that of the full 28-layer run; the evict launch covers 8 layers there and is scaled by the
+# layer count).  Set an entry to None when its kernel changes until the counters are taken again.
+NCU_DRAM_BYTES = {
+    "decode": 19.07e6,                 # one layer's K and V once (algorithmic: 18.9 MB)
+    "prefill": 22.94e6,                # one layer's K and V once plus Q and the output (the rest is served by L2)
+    "evict_per_layer": (71.4e6 + 15.4e6) / 8,   # reads all re-rotated keys; most of the write-back is still in L2 at kernel end
+}
+
+
 def prefill_flops(wl, n_q, lk):
     pairs = n_q * (lk - n_q) + n_q * (n_q + 1) // 2
     return 4 * wl.q_heads * wl.head_dim * pairs
@@ -404,8 +415,14 @@ def main():
         kernels[k]["frac"] = kernels[k]["achieved"] / kernels[k]["peak"]
     dominant = max(("prefill", "decode", "evict"), key=lambda k: kernels[k]["per_step_ms"])
     kd = kernels[dominant]
+    traffic = NCU_DRAM_BYTES.get(dominant)
+    if dominant == "evict" and NCU_DRAM_BYTES.get("evict_per_layer") is not None:
+        traffic = NCU_DRAM_BYTES["evict_per_layer"] * wl.layers
+    if args.config not in (2, 3):
+        traffic = None          # the counters were taken on the config-3 shape
     roofline = dict(bound="tensor" if dominant == "prefill" else "hbm", kernel=dominant, achieved=kd["achieved"],
-                    peak=kd["peak"], unit=kd["unit"], frac=kd["frac"], traffic=None,
+                    peak=kd["peak"], unit=kd["unit"], frac=kd["frac"], traffic=traffic,
+                    algorithmic=(flops if dominant == "prefill" else kv_bytes_layer if dominant == "decode" else evict_bytes),
                     peak_source=peaks["source"] + (" (burst bf16)" if dominant == "prefill" else " (copy)"))
 
     # ---- end to end through the host-buffer entry points -----------------------------------------
