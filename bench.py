@@ -212,6 +212,22 @@ NCU_DRAM_BYTES = {
 }
 
 
+def max_over_ranks(value: float, world: int, device="cuda") -> float:
+    """The slowest rank's figure (replicas run independent streams; the job is as slow as its slowest rank)."""
+    if world <= 1:
+        return float(value)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(world: int, units_per_step: float, ms_per_step: float) -> float:
+    """Units per second over all ranks: every rank processes `units_per_step` per step (weak scaling)."""
+    return world * units_per_step / (ms_per_step * 1e-3)
+
+
 def prefill_flops(wl, n_q, lk):
     pairs = n_q * (lk - n_q) + n_q * (n_q + 1) // 2
     return 4 * wl.q_heads * wl.head_dim * pairs
@@ -437,18 +453,12 @@ def main():
             run_step_host(cache, wl, hin[1 + i % 2])
         torch.cuda.synchronize()
         e2e_s = (time.perf_counter() - t0) / e2e_steps
-        if world > 1:
-            t = torch.tensor([e2e_s], device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_s = float(t.item())
-        e2e = dict(value=world * frames_per_step / e2e_s, unit="frames/s", ms_per_step=e2e_s * 1e3,
+        e2e_s = max_over_ranks(e2e_s, world)
+        e2e = dict(value=whole_job_value(world, frames_per_step, e2e_s * 1e3), unit="frames/s", ms_per_step=e2e_s * 1e3,
                    h2d_bytes_per_step=hin[1].h2d_bytes(), d2h_bytes_per_step=hin[1].d2h_bytes(),
                    api="svlm_cache_append_host / svlm_attend_host, all layers per call, pinned host buffers")
 
-    if world > 1:
-        t = torch.tensor([elapsed_ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        elapsed_ms = float(t.item())
+    elapsed_ms = max_over_ranks(elapsed_ms, world)
     ms_per_step = elapsed_ms / args.steps
 
     cpu = None
@@ -460,7 +470,7 @@ def main():
 
     if rank == 0:
         third = max(1, args.steps // 3)
-        line = dict(base, value=world * frames_per_step / (ms_per_step * 1e-3), ms_per_step=ms_per_step, config=config,
+        line = dict(base, value=whole_job_value(world, frames_per_step, ms_per_step), ms_per_step=ms_per_step, config=config,
                     roofline=roofline, cpu_baseline=cpu, e2e=e2e, gpu_launches=int(gpu_launches), clocks=clocks,
                     kernels=kernels, decode_tok_s=wl.decode_steps / (tot["decode_token"] * 1e-3),
                     step_ms=dict(min=min(step_ms), median=statistics.median(step_ms), max=max(step_ms),
