@@ -278,6 +278,104 @@ def oracle_sample(wl, rows=48, decode=2):
                        f"decode steps of one steady-state chunk; scaled linearly to the full step")
 
 
+def bench_batched_decode(args, wl, base, peaks, rank, world, local):
+    """Workload 4: `wl.streams` independent streams at the full retained size; a step is one batched q=1 decode step
+    (every stream appends its token, ONE attention launch serves all streams); the caches are evicted every 16 steps.
+    Whole cycles of 16 steps + evictions are replayed from a CUDA graph; value = decode tokens/s over all streams."""
+    import torch
+    from paper_2510_09608_b200 import binding
+    cycle = 16
+    streams = [sg.Stream(wl, rank * wl.streams + i) for i in range(wl.streams)]
+    caches = []
+    for st in streams:
+        c = binding.Cache(wl.layers, wl.kv_heads, wl.head_dim, wl.n_sink, wl.vision_window, wl.text_window, wl.capacity)
+        c.set_rope(wl.rope_mode, wl.rope_base, wl.sections)
+        fill_to_steady_state(c, dataclasses_replace(wl, decode_steps=cycle), st)
+        c.evict()
+        caches.append(c)
+
+    def make_cycle():
+        steps = []
+        for _ in range(cycle):
+            toks = [st.next_decode_token() for st in streams]
+            gen = lambda tensor, heads: torch.stack([sg.rows_bf16_torch(wl.seed, tensor, st.stream, 0, t[0], heads, wl.head_dim)  # noqa: E731
+                                                     for st, t in zip(streams, toks)])
+            steps.append(dict(K=gen(sg.TENSOR_K, wl.kv_heads), V=gen(sg.TENSOR_V, wl.kv_heads), Q=gen(sg.TENSOR_Q, wl.q_heads),
+                              types=torch.zeros(len(streams), 1, dtype=torch.uint8, device="cuda"),
+                              pos=torch.from_numpy(np.stack([t[2] for t in toks])).cuda()))
+            steps[-1]["out"] = torch.empty_like(steps[-1]["Q"])
+        return steps
+
+    def run_cycle(steps, timers=None):
+        for d in steps:
+            for i, c in enumerate(caches):
+                c.append(0, d["K"][i], d["V"][i], d["types"][i], d["pos"][i])
+            if timers is not None:
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record()
+            binding.attend_batched(caches, 0, d["Q"], d["pos"], d["out"])
+            if timers is not None:
+                b.record()
+                timers.append((a, b))
+        for c in caches:
+            c.evict()
+
+    n_cycles = max(1, (args.warmup + args.steps + cycle - 1) // cycle) + 1
+    cycles = [make_cycle() for _ in range(n_cycles)]
+    run_cycle(cycles[0])                      # plain once: one-time kernel attributes outside any capture
+    torch.cuda.synchronize()
+    graphs = []
+    cur = torch.cuda.current_stream()
+    for cy in cycles[1:]:
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            for c in caches:
+                c.set_stream(torch.cuda.current_stream())
+            run_cycle(cy)
+        graphs.append(g)
+    for c in caches:
+        c.set_stream(cur)
+    graphs[0].replay()                        # warm-up cycle (>= 3 steps)
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local)
+    sampler.start()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    before = binding.launch_count()
+    ev0.record()
+    for g in graphs[1:] or graphs:
+        g.replay()
+    ev1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.finish()
+    timed_cycles = len(graphs[1:] or graphs)
+    ms_per_step = max_over_ranks(ev0.elapsed_time(ev1), world) / (timed_cycles * cycle)
+    launches = (cycle * (2 * len(caches) + 1) + 2 * len(caches)) * timed_cycles
+    timers = []
+    run_cycle(make_cycle(), timers)
+    torch.cuda.synchronize()
+    att_ms = statistics.median(a.elapsed_time(b) for a, b in timers)
+    for c in caches:
+        assert c.status() == binding.OK
+    kv_bytes = wl.retained * 2 * wl.kv_heads * wl.head_dim * 2 * len(caches)
+    roof = dict(bound="hbm", kernel="decode (batched)", achieved=kv_bytes / (att_ms * 1e-3) / 1e9, peak=peaks["hbm"], unit="GB/s",
+                traffic=None, algorithmic=kv_bytes, avg_ms=att_ms, peak_source=peaks["source"] + " (copy)")
+    roof["frac"] = roof["achieved"] / roof["peak"]
+    if rank == 0:
+        print(json.dumps(dict(base, metric="decode tokens/s, batched q=1 steps with interleaved eviction", unit="tok/s",
+                              value=whole_job_value(world, len(caches), ms_per_step), ms_per_step=ms_per_step,
+                              config=dict(workload=f"config 4 ({wl.name}): {len(caches)} streams x {wl.layers} layer, {wl.q_heads}/"
+                                                   f"{wl.kv_heads} heads, d={wl.head_dim}, retained {wl.retained} tokens per stream, "
+                                                   f"evict every {cycle} steps", l2="302 MB of K/V per step, above L2; no flush",
+                                          replicas="independent streams per GPU, no collective"),
+                              roofline=roof, cpu_baseline=None, e2e=None, gpu_launches=int(launches), clocks=clocks,
+                              steps=timed_cycles * cycle)))
+
+
+def dataclasses_replace(obj, **kw):
+    import dataclasses
+    return dataclasses.replace(obj, **kw)
+
+
 # ------------------------------------------------------------------------------------------------
 def main():
     ap = argparse.ArgumentParser()
@@ -341,6 +439,11 @@ def main():
         torch.cuda.synchronize()
 
     peaks = load_peaks()
+    if wl.streams > 1 and wl.layers == 1:
+        bench_batched_decode(args, wl, base, peaks, rank, world, local)
+        if world > 1:
+            dist.destroy_process_group()
+        return
     stream = sg.Stream(wl, rank)
     cache = binding.Cache(wl.layers, wl.kv_heads, wl.head_dim, wl.n_sink, wl.vision_window, wl.text_window, wl.capacity)
     cache.set_rope(wl.rope_mode, wl.rope_base, wl.sections)

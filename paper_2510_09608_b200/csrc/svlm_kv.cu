@@ -6,6 +6,7 @@
 #include <cuda_runtime.h>
 #include "svlm_dev.h"
 #include "svlm_launch.h"
+#include "svlm_rope.cuh"
 
 namespace {
 
@@ -28,7 +29,7 @@ __device__ __forceinline__ void rotate8(Bf16x8& lo, Bf16x8& hi, const float* cs,
 }
 
 // One thread per (token, group of 8 pairs); it serves every kv head (and every layer when
-// layer < 0) of that token, so the sines are computed once.  Angles are formed in fp64.
+// layer < 0) of that token, so the rotation factors are looked up once (table, see svlm_rope.cuh).
 __global__ void __launch_bounds__(256) kv_write_kernel(SvlmCacheDev cd, int layer, const uint16_t* __restrict__ K,
                                                        const uint16_t* __restrict__ V, int n) {
     if (cd.ctrl->append_n != n) return;   // the metadata append was dropped (capacity) or does not match
@@ -47,10 +48,10 @@ __global__ void __launch_bounds__(256) kv_write_kernel(SvlmCacheDev cd, int laye
     for (int j = 0; j < 8; ++j) {
         const int pair = g * 8 + j;
         const int axis = cd.rope_mode == 0 ? 0 : (pair < cd.sec_t ? 0 : (pair < cd.sec_th ? 1 : 2));
-        double s, c;
-        sincos((double)cd.slot_c[axis * cd.n_slots + slot] * cd.theta[pair], &s, &c);
-        cs[j] = (float)c;
-        sn[j] = (float)s;
+        const float2 f = svlm_rope_cs(reinterpret_cast<const float2*>(cd.rope_tab), half, pair,
+                                      cd.slot_c[axis * cd.n_slots + slot], cd.theta[pair]);
+        cs[j] = f.x;
+        sn[j] = f.y;
     }
     const int d = cd.head_dim;
     const int l0 = layer < 0 ? 0 : layer, l1 = layer < 0 ? cd.layers : layer + 1;
@@ -88,10 +89,10 @@ __global__ void __launch_bounds__(256) evict_rotate_kernel(SvlmCacheDev cd, int 
     float cs[8], sn[8];
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
-        double s, c;
-        sincos(-(double)delta * cd.theta[g * 8 + j], &s, &c);
-        cs[j] = (float)c;
-        sn[j] = (float)s;
+        const float2 f = svlm_rope_cs(reinterpret_cast<const float2*>(cd.rope_tab), half, g * 8 + j, -(long long)delta,
+                                      cd.theta[g * 8 + j]);
+        cs[j] = f.x;
+        sn[j] = f.y;
     }
     const int d = cd.head_dim;
     const int row0 = blockIdx.y * layers_per_block * cd.kv_heads;
