@@ -208,3 +208,52 @@ def test_config5_high_frame_rate_streams_sampled():
             _close(dev_to_f64(inp.dec[-1]["out"][l]), ref.attend(l, stream.q(l, g1), p1), f"stream {sid} last decode layer {l}")
         _same_metadata(cache, ref)
         _check_kv(cache, ref, stream, wl, 3, n_evicts + 1)
+
+
+def test_config2_whole_600_chunk_stream_metadata_and_final_outputs():
+    """The complete 600-chunk single-layer stream (ten minutes at one chunk per second, 16 generated tokens per
+    chunk): ring ordinals, page tables and positions run far past their first wrap.  Kept ordinals, positions
+    and total shift are compared bit-exactly every 50 chunks; stored keys and attention outputs at the end."""
+    from harness import bits_to_dev, dev_to_f64
+    from paper_2510_09608_b200 import streamgen as sg
+    wl = sg.workloads()[2]
+    stream, cache, ref = _setup(wl)
+    gen = lambda tensor, g, heads: sg.rows_bf16_torch(wl.seed, tensor, 0, 0, g, heads, wl.head_dim)  # noqa: E731
+    n_evicts = 0
+    max_pos = 0
+    for chunk in range(wl.chunks):
+        gids, types, pos = stream.next_chunk()
+        cache.append(0, gen(sg.TENSOR_K, gids, wl.kv_heads), gen(sg.TENSOR_V, gids, wl.kv_heads),
+                     torch.from_numpy(types).cuda(), torch.from_numpy(np.ascontiguousarray(pos)).cuda())
+        cache.evict()
+        ref.append(None, None, types, pos)
+        ref.evict()
+        n_evicts += 1
+        toks = [stream.next_decode_token() for _ in range(wl.decode_steps)]
+        g = np.concatenate([t[0] for t in toks]); ty = np.concatenate([t[1] for t in toks]); p = np.concatenate([t[2] for t in toks])
+        last = chunk == wl.chunks - 1
+        if not last:      # generated tokens in bulk: the same metadata as sixteen single appends
+            cache.append(0, gen(sg.TENSOR_K, g, wl.kv_heads), gen(sg.TENSOR_V, g, wl.kv_heads), torch.from_numpy(ty).cuda(),
+                         torch.from_numpy(np.ascontiguousarray(p)).cuda())
+            ref.append(None, None, ty, p)
+        if chunk % 50 == 49 or last:
+            _same_metadata(cache, ref)
+            max_pos = max(max_pos, int(ref.query()["pos"].max()))
+    # bounded positions (contiguous RoPE): never beyond retained tokens + one chunk's span
+    assert max_pos < wl.n_sink + wl.text_window + wl.vision_window + wl.max_chunk_tokens + wl.decode_steps
+    # the last chunk: prefill rows and fused decode steps against the checker
+    _give(ref, stream, 0)
+    rng = np.random.default_rng(wl.seed)
+    rows = np.unique(np.concatenate([[0, len(gids) - 1], rng.integers(0, len(gids), 16)]))
+    qp = torch.from_numpy(np.ascontiguousarray(pos)).cuda()
+    out = dev_to_f64(cache.attend(0, gen(sg.TENSOR_Q, gids, wl.q_heads), qp))
+    _close(out[rows], ref.attend(0, stream.q(0, gids), pos, rows), "last chunk prefill")
+    for g1, t1, p1 in toks:
+        o = dev_to_f64(cache.decode_step(0, bits_to_dev(stream.k(0, g1)), bits_to_dev(stream.v(0, g1)),
+                                         torch.from_numpy(t1).cuda(), torch.from_numpy(np.ascontiguousarray(p1)).cuda(),
+                                         bits_to_dev(stream.q(0, g1))))
+        ref.append(None, None, t1, p1)
+        _give_new(ref, stream, 0, g1)
+        _close(o, ref.attend(0, stream.q(0, g1), p1), "decode after 600 chunks")
+    _same_metadata(cache, ref)
+    _check_kv(cache, ref, stream, wl, 0, n_evicts)
