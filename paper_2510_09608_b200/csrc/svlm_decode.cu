@@ -210,17 +210,23 @@ decode_kernel(SvlmAttendBatch b, int layer0, int n_layers, const uint16_t* __res
                 const int* qp = q_pos + (size_t)ci * (b.rope_mode == 0 ? 1 : 3);
                 cs = svlm_rope_cs(tab, HALF, pair, (long long)qp[b.rope_mode == 0 ? 0 : axis] - shift, b.theta[pair]);
             }
-            for (int h = threadIdx.x / HALF; h < 8; h += (DEC_CWARPS * 32) / HALF) {
-                float lo = 0.f, hi = 0.f;
-                if (h < G) {
-                    const size_t off = (((size_t)prob) * q_heads + hk * G + h) * D;   // n_q = 1
-                    const float x = __bfloat162float(__ushort_as_bfloat16(Q[off + pair]));
-                    const float y = __bfloat162float(__ushort_as_bfloat16(Q[off + pair + HALF]));
-                    lo = x * cs.x - y * cs.y;
-                    hi = y * cs.x + x * cs.y;
-                }
-                s_q[h * D + pair] = __bfloat16_as_ushort(__float2bfloat16_rn(lo));
-                s_q[h * D + pair + HALF] = __bfloat16_as_ushort(__float2bfloat16_rn(hi));
+            constexpr int HSTEP = (DEC_CWARPS * 32) / HALF, HN = (8 + HSTEP - 1) / HSTEP;   // heads per thread
+            uint16_t qx[HN], qy[HN];
+#pragma unroll
+            for (int k = 0; k < HN; ++k) {      // all loads first: one round trip
+                const int h = threadIdx.x / HALF + k * HSTEP;
+                const size_t off = (((size_t)prob) * q_heads + hk * G + (h < G ? h : 0)) * D;   // n_q = 1
+                qx[k] = Q[off + pair];
+                qy[k] = Q[off + pair + HALF];
+            }
+#pragma unroll
+            for (int k = 0; k < HN; ++k) {
+                const int h = threadIdx.x / HALF + k * HSTEP;
+                if (h >= 8) continue;
+                const float x = h < G ? __bfloat162float(__ushort_as_bfloat16(qx[k])) : 0.f;
+                const float y = h < G ? __bfloat162float(__ushort_as_bfloat16(qy[k])) : 0.f;
+                s_q[h * D + pair] = __bfloat16_as_ushort(__float2bfloat16_rn(x * cs.x - y * cs.y));
+                s_q[h * D + pair + HALF] = __bfloat16_as_ushort(__float2bfloat16_rn(y * cs.x + x * cs.y));
             }
         }
         asm volatile("bar.sync 1, %0;" ::"n"(DEC_CWARPS * 32));   // consumer warps only
