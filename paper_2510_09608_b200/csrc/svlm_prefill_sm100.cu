@@ -345,66 +345,88 @@ prefill_kernel(SvlmAttendBatch b, int layer0, int n_layers, const uint16_t* __re
 #pragma unroll
             for (int u = 0; u < UN; ++u) {
                 const int i = base + u * PF_THREADS + threadIdx.x;
-                if (i < n_ent) s_cs[i] = svlm_rope_cs(tab, HALF, i % HALF, cpos[u], b.theta[i % HALF]);
+                if (i < n_ent) {
+                    // a token's factors are read back 64 bytes per thread at a 64-byte lane stride: the 16-byte
+                    // chunks are XOR-swizzled so that eight such lanes hit eight different bank groups
+                    const int tk = i / HALF, pair = i % HALF;
+                    s_cs[tk * HALF + ((((pair >> 1) ^ (pair >> 4)) << 1) | (pair & 1))] =
+                        svlm_rope_cs(tab, HALF, pair, cpos[u], b.theta[pair]);
+                }
             }
         }
     }
     __syncthreads();
-    // (2) every softmax thread rotates its own row
+    // (2) rotation of the 256 rows, coalesced: a work item is (row, chunk c of 8 pairs) = the 16-byte chunk c of the
+    //     row's low half with its partner chunk of the high half; consecutive threads take consecutive chunks of a
+    //     row, so global loads and factor look-ups of a warp touch few lines and several items are in flight.
     if (warp < 8) {
-        const int g = warp >> 2, m = threadIdx.x & 127;
-        const int mg = m0 + g * 128 + m;
-        const bool live = mg < m_total;
-        const int r = live ? mg / G : r_lo, h = live ? mg % G : 0;
-        const uint16_t* src = Q + ((((size_t)prob) * n_q + r) * q_heads + hk * G + h) * D;
-        const float2* cs_row = s_cs + (size_t)(r - r_lo) * HALF;
-        const int* qp = q_pos + ((size_t)ci * n_q + r) * (b.rope_mode == 0 ? 1 : 3);
-        unsigned char* sQg = sQ + g * TILE_BYTES;
-        // (a compact loop: the code runs once per thread, so its instruction footprint matters more than its
-        //  schedule; the next chunk's loads are issued before the current chunk is rotated)
-        auto ld_chunk = [&](int i) { return live ? __ldg(reinterpret_cast<const uint4*>(src) + i) : make_uint4(0, 0, 0, 0); };
-        uint4 lo_n = ld_chunk(0), hi_n = ld_chunk(HALF / 8);
-#pragma unroll 2
-        for (int c8 = 0; c8 < HALF / 8; ++c8) {    // 8 pairs at a time: chunk c8 of the low half, same of the high half
-            const uint4 lo4 = lo_n, hi4 = hi_n;
-            if (c8 + 1 < HALF / 8) { lo_n = ld_chunk(c8 + 1); hi_n = ld_chunk(HALF / 8 + c8 + 1); }
-            const unsigned* lw = reinterpret_cast<const unsigned*>(&lo4);
-            const unsigned* hw = reinterpret_cast<const unsigned*>(&hi4);
-            float2 cs8[8];
-            if (cs_shared) {
-#pragma unroll
-                for (int i = 0; i < 8; ++i) cs8[i] = cs_row[c8 * 8 + i];
-            } else {
+        constexpr int CH = HALF / 8;               // chunks per half row
+        constexpr int ITEMS = PF_ROWS * CH, PER = ITEMS / 256, UN = 4;
+        static_assert(PER % UN == 0, "items per thread");
 #pragma unroll 1
-                for (int i = 0; i < 8; ++i) {      // direct look-ups (too many tokens for the shared table)
-                    const int pair = c8 * 8 + i;
-                    const int axis = b.rope_mode == 0 ? 0 : (pair < b.sec_t ? 0 : (pair < b.sec_th ? 1 : 2));
-                    const float2 v = svlm_rope_cs(tab, HALF, pair, (long long)qp[b.rope_mode == 0 ? 0 : axis] - shift, b.theta[pair]);
+        for (int it0 = 0; it0 < PER; it0 += UN) {
+            uint4 lo4[UN], hi4[UN];
+            int row[UN], c8v[UN], tok[UN];
 #pragma unroll
-                    for (int q = 0; q < 8; ++q) if (q == i) cs8[q] = v;
-                }
+            for (int u = 0; u < UN; ++u) {         // all loads of the batch first
+                const int item = (it0 + u) * 256 + threadIdx.x;
+                row[u] = item / CH; c8v[u] = item % CH;
+                const int mg = m0 + row[u];
+                const bool live = mg < m_total;
+                const int r = live ? mg / G : r_lo, h = live ? mg % G : 0;
+                tok[u] = r;
+                const uint4* src = reinterpret_cast<const uint4*>(Q + ((((size_t)prob) * n_q + r) * q_heads + hk * G + h) * D);
+                lo4[u] = live ? __ldg(src + c8v[u]) : make_uint4(0, 0, 0, 0);
+                hi4[u] = live ? __ldg(src + CH + c8v[u]) : make_uint4(0, 0, 0, 0);
             }
-            unsigned lo_o[4], hi_o[4];
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                float xl[2] = {__uint_as_float(lw[j] << 16), __uint_as_float(lw[j] & 0xffff0000u)};
-                float xh[2] = {__uint_as_float(hw[j] << 16), __uint_as_float(hw[j] & 0xffff0000u)};
-                float ol[2], oh[2];
+            for (int u = 0; u < UN; ++u) {
+                const int c8 = c8v[u], g = row[u] >> 7, m = row[u] & 127;
+                const float2* cs_row = s_cs + (size_t)(tok[u] - r_lo) * HALF;
+                const int* qp = q_pos + ((size_t)ci * n_q + tok[u]) * (b.rope_mode == 0 ? 1 : 3);
+                const unsigned* lw = reinterpret_cast<const unsigned*>(&lo4[u]);
+                const unsigned* hw = reinterpret_cast<const unsigned*>(&hi4[u]);
+                float2 cs8[8];
+                if (cs_shared) {
 #pragma unroll
-                for (int e = 0; e < 2; ++e) {
-                    const float2 cs = cs8[2 * j + e];
-                    ol[e] = xl[e] * cs.x - xh[e] * cs.y;
-                    oh[e] = xh[e] * cs.x + xl[e] * cs.y;
+                    for (int j = 0; j < 4; ++j) {
+                        const float4 v = *reinterpret_cast<const float4*>(cs_row + (((4 * c8 + j) ^ (c8 >> 1)) << 1));
+                        cs8[2 * j] = make_float2(v.x, v.y);
+                        cs8[2 * j + 1] = make_float2(v.z, v.w);
+                    }
+                } else {
+#pragma unroll 1
+                    for (int i = 0; i < 8; ++i) {      // direct look-ups (too many tokens for the shared table)
+                        const int pair = c8 * 8 + i;
+                        const int axis = b.rope_mode == 0 ? 0 : (pair < b.sec_t ? 0 : (pair < b.sec_th ? 1 : 2));
+                        const float2 v = svlm_rope_cs(tab, HALF, pair, (long long)qp[b.rope_mode == 0 ? 0 : axis] - shift, b.theta[pair]);
+#pragma unroll
+                        for (int q = 0; q < 8; ++q) if (q == i) cs8[q] = v;
+                    }
                 }
-                lo_o[j] = pack2(ol[0], ol[1]);
-                hi_o[j] = pack2(oh[0], oh[1]);
+                unsigned lo_o[4], hi_o[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    float xl[2] = {__uint_as_float(lw[j] << 16), __uint_as_float(lw[j] & 0xffff0000u)};
+                    float xh[2] = {__uint_as_float(hw[j] << 16), __uint_as_float(hw[j] & 0xffff0000u)};
+                    float ol[2], oh[2];
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        const float2 cs = cs8[2 * j + e];
+                        ol[e] = xl[e] * cs.x - xh[e] * cs.y;
+                        oh[e] = xh[e] * cs.x + xl[e] * cs.y;
+                    }
+                    lo_o[j] = pack2(ol[0], ol[1]);
+                    hi_o[j] = pack2(oh[0], oh[1]);
+                }
+                // element e of the row lives in block e/64, 16-byte chunk (e%64)/8, XOR-swizzled by row&7
+                unsigned char* sQg = sQ + g * TILE_BYTES;
+                const int e_lo = c8 * 8, e_hi = HALF + c8 * 8;
+                unsigned char* dl = sQg + (e_lo / 64) * (128 * 128) + m * 128 + ((((e_lo % 64) / 8) ^ (m & 7)) << 4);
+                unsigned char* dh = sQg + (e_hi / 64) * (128 * 128) + m * 128 + ((((e_hi % 64) / 8) ^ (m & 7)) << 4);
+                *reinterpret_cast<uint4*>(dl) = make_uint4(lo_o[0], lo_o[1], lo_o[2], lo_o[3]);
+                *reinterpret_cast<uint4*>(dh) = make_uint4(hi_o[0], hi_o[1], hi_o[2], hi_o[3]);
             }
-            // element e of the row lives in block e/64, 16-byte chunk (e%64)/8, XOR-swizzled by row&7
-            const int e_lo = c8 * 8, e_hi = HALF + c8 * 8;
-            unsigned char* dl = sQg + (e_lo / 64) * (128 * 128) + m * 128 + ((((e_lo % 64) / 8) ^ (m & 7)) << 4);
-            unsigned char* dh = sQg + (e_hi / 64) * (128 * 128) + m * 128 + ((((e_hi % 64) / 8) ^ (m & 7)) << 4);
-            *reinterpret_cast<uint4*>(dl) = make_uint4(lo_o[0], lo_o[1], lo_o[2], lo_o[3]);
-            *reinterpret_cast<uint4*>(dh) = make_uint4(hi_o[0], hi_o[1], hi_o[2], hi_o[3]);
         }
     }
     fence_proxy_async();   // the query tiles feed the tensor core, the borrowed ring stages get TMA writes next
