@@ -151,6 +151,24 @@ int svlm_attend_batched(svlm_cache* const* caches, int n_caches, int layer, cons
                         int n_q, int q_heads, void* out);
 
 /*
+ * Batched forms for independent streams that advance in lock step (one generated token per stream per
+ * step, as in batched serving; the paper's policy is per stream, so each cache behaves exactly as under
+ * the single-cache calls).  Same requirements on the caches as svlm_attend_batched; a cache may appear
+ * only once.
+ *
+ * svlm_decode_step_batched = svlm_decode_step on every cache, one metadata launch (layer 0) and one
+ * attention launch for all of them:
+ *   K, V        bf16 [n_caches][kv_heads][head_dim]      Q, out   bf16 [n_caches][q_heads][head_dim]
+ *   token_type  uint8 [n_caches]      pos   int32 [n_caches] or [n_caches][3]
+ * svlm_cache_evict_batched = svlm_cache_evict on every cache, one metadata launch and one re-rotation
+ * launch for all of them.
+ * Errors: as the single-cache calls; SVLM_ERR_ARG also for mismatched or repeated caches.
+ */
+int svlm_decode_step_batched(svlm_cache* const* caches, int n_caches, int layer, const void* K, const void* V,
+                             const uint8_t* token_type, const int32_t* pos, const void* Q, int q_heads, void* out);
+int svlm_cache_evict_batched(svlm_cache* const* caches, int n_caches);
+
+/*
  * Host-buffer variants: the same operations with K, V, token_type, pos / Q, q_pos, out in HOST
  * memory (pinned memory makes the copies asynchronous).  The library stages them through device
  * buffers it owns (grown on demand, which synchronises once).  svlm_attend_host returns after the

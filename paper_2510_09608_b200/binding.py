@@ -36,6 +36,8 @@ _lib.svlm_cache_evict.argtypes = [_vp]
 _lib.svlm_attend.argtypes = [_vp, _i, _vp, _vp, _i, _i, _vp]
 _lib.svlm_decode_step.argtypes = [_vp, _i, _vp, _vp, _vp, _vp, _vp, _i, _vp]
 _lib.svlm_attend_batched.argtypes = [C.POINTER(_vp), _i, _i, _vp, _vp, _i, _i, _vp]
+_lib.svlm_decode_step_batched.argtypes = [C.POINTER(_vp), _i, _i, _vp, _vp, _vp, _vp, _vp, _i, _vp]
+_lib.svlm_cache_evict_batched.argtypes = [C.POINTER(_vp), _i]
 _lib.svlm_cache_append_host.argtypes = [_vp, _i, _vp, _vp, _vp, _vp, _i]
 _lib.svlm_attend_host.argtypes = [_vp, _i, _vp, _vp, _i, _i, _vp]
 _lib.svlm_attend_decode_noalloc.argtypes = [_vp, _i, _vp, _vp, _i, _vp]
@@ -201,3 +203,21 @@ def attend_batched(caches, layer, Q, q_pos, out=None):
                                   Q.shape[1], Q.shape[2], _dev_ptr(out, torch.bfloat16))
     _check(rc, "svlm_attend_batched")
     return out
+
+
+def decode_step_batched(caches, layer, K, V, token_type, pos, Q, out=None):
+    """One generated token per cache: K, V [n_caches, kv_heads, d], Q [n_caches, q_heads, d] bf16 CUDA, token_type
+    uint8 [n_caches], pos int32 [n_caches] or [n_caches, 3]; one launch for all caches (svlm_decode_step_batched)."""
+    if out is None:
+        out = torch.empty_like(Q)
+    arr = (_vp * len(caches))(*[c._h for c in caches])
+    rc = _lib.svlm_decode_step_batched(arr, len(caches), layer, _dev_ptr(K, torch.bfloat16), _dev_ptr(V, torch.bfloat16),
+                                       _dev_ptr(token_type, torch.uint8), _dev_ptr(pos, torch.int32),
+                                       _dev_ptr(Q, torch.bfloat16), Q.shape[-2], _dev_ptr(out, torch.bfloat16))
+    _check(rc, "svlm_decode_step_batched")
+    return out
+
+
+def evict_batched(caches):
+    arr = (_vp * len(caches))(*[c._h for c in caches])
+    _check(_lib.svlm_cache_evict_batched(arr, len(caches)), "svlm_cache_evict_batched")

@@ -72,6 +72,21 @@ struct SvlmCacheDev {        // passed by value to kernels
     double theta[SVLM_MAX_HALF];   // base^(-2i/head_dim)
 };
 
+struct SvlmCacheList {       // kernel parameter of the batched metadata and re-rotation kernels
+    int n;
+    const SvlmCacheDev* cd[SVLM_MAX_BATCH];   // the caches' descriptors, copies in device memory
+};
+
+#ifdef __CUDACC__
+// All threads of the block copy a descriptor from device memory to shared memory and synchronise.
+__device__ __forceinline__ void svlm_load_desc(SvlmCacheDev* dst, const SvlmCacheDev* src) {
+    static_assert(sizeof(SvlmCacheDev) % 4 == 0, "descriptor is copied in 32-bit words");
+    for (int i = threadIdx.x; i < (int)(sizeof(SvlmCacheDev) / 4); i += blockDim.x)
+        reinterpret_cast<int*>(dst)[i] = reinterpret_cast<const int*>(src)[i];
+    __syncthreads();
+}
+#endif
+
 struct SvlmAttendView {      // what attention needs from one cache
     const uint16_t* K;
     const uint16_t* V;

@@ -77,7 +77,7 @@ __global__ void __launch_bounds__(256) kv_write_kernel(SvlmCacheDev cd, int laye
 // the angle -E*theta is identical on the three MRoPE axes because all three indices of a token
 // shift by the same E.
 template <int UNROLL>
-__global__ void __launch_bounds__(256) evict_rotate_kernel(SvlmCacheDev cd, int layers_per_block) {
+__device__ __forceinline__ void evict_rotate_body(const SvlmCacheDev& cd, int layers_per_block) {
     if (!cd.ctrl->evict_moved) return;
     const int half = cd.head_dim / 2;
     const int groups = half / 8;
@@ -117,6 +117,26 @@ __global__ void __launch_bounds__(256) evict_rotate_kernel(SvlmCacheDev cd, int 
     }
 }
 
+template <int UNROLL>
+__global__ void __launch_bounds__(256) evict_rotate_kernel(SvlmCacheDev cd, int layers_per_block) {
+    evict_rotate_body<UNROLL>(cd, layers_per_block);
+}
+
+// Batched form: blockIdx.z selects the cache, whose descriptor is first copied to shared memory.
+template <int UNROLL>
+__global__ void __launch_bounds__(256) evict_rotate_batch_kernel(SvlmCacheList list, int layers_per_block) {
+    __shared__ SvlmCacheDev s_cd;
+    svlm_load_desc(&s_cd, list.cd[blockIdx.z]);
+    evict_rotate_body<UNROLL>(s_cd, layers_per_block);
+}
+
+// Layers per block in y: enough blocks to fill the machine a few times over, at least 4 rows per thread.
+int rotate_layers_per_block(int layers, int kv_heads) {
+    int splits = 1;
+    while (splits < layers && (layers + splits - 1) / splits * kv_heads > 8) ++splits;
+    return (layers + splits - 1) / splits;
+}
+
 }  // namespace
 
 void svlm_launch_kv_write(const SvlmCacheDev& cd, int layer, const void* K, const void* V, int n, cudaStream_t st) {
@@ -129,11 +149,16 @@ void svlm_launch_kv_write(const SvlmCacheDev& cd, int layer, const void* K, cons
 void svlm_launch_evict_rotate(const SvlmCacheDev& cd, cudaStream_t st) {
     const int groups = cd.head_dim / 16;
     const int threads = cd.n_slots * groups;
-    // enough blocks in y to fill the machine a few times over, at least 4 rows per thread
-    int splits = 1;
-    while (splits < cd.layers && (cd.layers + splits - 1) / splits * cd.kv_heads > 8) ++splits;
-    const int lpb = (cd.layers + splits - 1) / splits;
+    const int lpb = rotate_layers_per_block(cd.layers, cd.kv_heads);
     dim3 grid((threads + 255) / 256, (cd.layers + lpb - 1) / lpb);
     evict_rotate_kernel<4><<<grid, 256, 0, st>>>(cd, lpb);
+    svlm_count_launch();
+}
+
+void svlm_launch_evict_rotate_batch(const SvlmCacheList& list, const SvlmCacheDev& geom, cudaStream_t st) {
+    const int threads = geom.n_slots * (geom.head_dim / 16);
+    const int lpb = rotate_layers_per_block(geom.layers, geom.kv_heads);
+    dim3 grid((threads + 255) / 256, (geom.layers + lpb - 1) / lpb, list.n);
+    evict_rotate_batch_kernel<4><<<grid, 256, 0, st>>>(list, lpb);
     svlm_count_launch();
 }

@@ -8,11 +8,17 @@ void svlm_count_launch();
 // metadata (svlm_meta.cu)
 void svlm_launch_append_meta(const SvlmCacheDev& cd, const unsigned char* types, const int* pos, int n, cudaStream_t st);
 void svlm_launch_evict_meta(const SvlmCacheDev& cd, cudaStream_t st);
+// batched forms, one block per cache: types [n_caches][n], pos [n_caches][n](x3)
+void svlm_launch_append_meta_batch(const SvlmCacheList& list, const unsigned char* types, const int* pos, int n,
+                                   cudaStream_t st);
+void svlm_launch_evict_meta_batch(const SvlmCacheList& list, cudaStream_t st);
 
 // key/value movement (svlm_kv.cu)
 // layer < 0: K,V are [layers][n][kv_heads][d]; otherwise [n][kv_heads][d] for that layer.
 void svlm_launch_kv_write(const SvlmCacheDev& cd, int layer, const void* K, const void* V, int n, cudaStream_t st);
 void svlm_launch_evict_rotate(const SvlmCacheDev& cd, cudaStream_t st);
+// every cache of the list has the geometry of geom
+void svlm_launch_evict_rotate_batch(const SvlmCacheList& list, const SvlmCacheDev& geom, cudaStream_t st);
 
 // attention (svlm_attend_simple.cu)
 // Q, out: [n_caches][n_layers][n_q][q_heads][d]; q_pos: [n_caches][n_q](x3)

@@ -144,8 +144,8 @@ __device__ void rebuild_tiles(const SvlmCacheDev& cd, int sink_fill, const long 
 // ---------------------------------------------------------------------------------------------
 // Append: stream ordinal, per-type ordinal, cursor advance a = max(0, max(p)+1 - cursor),
 // contiguous position c = p - shift_total, and the storage slot of each of the n new tokens.
-__global__ void __launch_bounds__(META_THREADS) append_meta_kernel(SvlmCacheDev cd, const unsigned char* types,
-                                                                   const int* pos, int n) {
+__device__ __forceinline__ void append_meta_body(const SvlmCacheDev& cd, const unsigned char* types, const int* pos,
+                                                 int n) {
     __shared__ int wbuf[META_WARPS];
     __shared__ long long wbuf64[META_WARPS];
     __shared__ int s_cnt[3];     // text tokens; sink tokens of type TEXT / VISION in this append
@@ -282,7 +282,7 @@ __device__ __forceinline__ int count_below(const long long* g, int n, long long 
 // Evict: keep-mask (a suffix of each ring plus the sinks), prefix sums of the evicted tokens'
 // cursor advances, and the left-shift E(i) of every retained token i: the advances of all evicted
 // tokens that precede it in the stream.
-__global__ void __launch_bounds__(META_THREADS) evict_meta_kernel(SvlmCacheDev cd) {
+__device__ __forceinline__ void evict_meta_body(const SvlmCacheDev& cd) {
     __shared__ long long wbuf64[META_WARPS];
     __shared__ int s_moved;
     SvlmCtrl* ctrl = cd.ctrl;
@@ -368,7 +368,40 @@ __global__ void __launch_bounds__(META_THREADS) evict_meta_kernel(SvlmCacheDev c
     }
 }
 
+__global__ void __launch_bounds__(META_THREADS) append_meta_kernel(SvlmCacheDev cd, const unsigned char* types,
+                                                                   const int* pos, int n) {
+    append_meta_body(cd, types, pos, n);
+}
+
+__global__ void __launch_bounds__(META_THREADS) evict_meta_kernel(SvlmCacheDev cd) { evict_meta_body(cd); }
+
+// Batched forms: block i serves cache i, whose descriptor it first copies from device memory into
+// shared memory.  types is [n_caches][n], pos [n_caches][n] (1D) or [n_caches][n][3].
+__global__ void __launch_bounds__(META_THREADS) append_meta_batch_kernel(SvlmCacheList list, const unsigned char* types,
+                                                                         const int* pos, int n) {
+    __shared__ SvlmCacheDev s_cd;
+    svlm_load_desc(&s_cd, list.cd[blockIdx.x]);
+    append_meta_body(s_cd, types + (size_t)blockIdx.x * n, pos + (size_t)blockIdx.x * n * (s_cd.rope_mode == 0 ? 1 : 3), n);
+}
+
+__global__ void __launch_bounds__(META_THREADS) evict_meta_batch_kernel(SvlmCacheList list) {
+    __shared__ SvlmCacheDev s_cd;
+    svlm_load_desc(&s_cd, list.cd[blockIdx.x]);
+    evict_meta_body(s_cd);
+}
+
 }  // namespace
+
+void svlm_launch_append_meta_batch(const SvlmCacheList& list, const unsigned char* types, const int* pos, int n,
+                                   cudaStream_t st) {
+    append_meta_batch_kernel<<<list.n, META_THREADS, 0, st>>>(list, types, pos, n);
+    svlm_count_launch();
+}
+
+void svlm_launch_evict_meta_batch(const SvlmCacheList& list, cudaStream_t st) {
+    evict_meta_batch_kernel<<<list.n, META_THREADS, 0, st>>>(list);
+    svlm_count_launch();
+}
 
 void svlm_launch_append_meta(const SvlmCacheDev& cd, const unsigned char* types, const int* pos, int n,
                              cudaStream_t st) {

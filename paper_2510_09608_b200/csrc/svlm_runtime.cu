@@ -135,6 +135,34 @@ void fill_batch_geometry(const svlm_cache* c, SvlmAttendBatch& b) {
     b.rope_tab = c->dev.rope_tab;
 }
 
+// Caches that may share one launch: same shape, rotary settings and device.
+bool same_geometry(const svlm_cache* c, const svlm_cache* c0) {
+    return c->dev.layers == c0->dev.layers && c->dev.kv_heads == c0->dev.kv_heads &&
+           c->dev.head_dim == c0->dev.head_dim && c->dev.n_slots == c0->dev.n_slots &&
+           c->dev.rope_mode == c0->dev.rope_mode && c->dev.sec_t == c0->dev.sec_t && c->dev.sec_th == c0->dev.sec_th &&
+           c->dev.theta[1] == c0->dev.theta[1] && c->device == c0->device;
+}
+
+// The descriptor copy in device memory that the batched kernels read (refreshed by every call that
+// changes the configuration; the configuration is frozen by the first append).
+int sync_dev_copy(svlm_cache* c) {
+    if (cudaMemcpy(c->dev_copy, &c->dev, sizeof(SvlmCacheDev), cudaMemcpyHostToDevice) != cudaSuccess) return SVLM_ERR_CUDA;
+    return SVLM_OK;
+}
+
+// Kernel parameter naming the caches of a batched call; all must be distinct and share a geometry.
+int make_list(svlm_cache* const* caches, int n_caches, SvlmCacheList& list) {
+    if (!caches || n_caches < 1 || n_caches > SVLM_MAX_BATCH || !caches[0]) return SVLM_ERR_ARG;
+    list.n = n_caches;
+    for (int i = 0; i < n_caches; ++i) {
+        if (!caches[i] || !same_geometry(caches[i], caches[0])) return SVLM_ERR_ARG;
+        for (int j = 0; j < i; ++j)
+            if (caches[j] == caches[i]) return SVLM_ERR_ARG;
+        list.cd[i] = caches[i]->dev_copy;
+    }
+    return SVLM_OK;
+}
+
 int attend_common(svlm_cache* const* caches, int n_caches, int layer, const void* Q, const int32_t* q_pos, int n_q,
                   int q_heads, void* out, const void* Knew = nullptr, const void* Vnew = nullptr) {
     svlm_cache* c0 = caches[0];
@@ -147,11 +175,7 @@ int attend_common(svlm_cache* const* caches, int n_caches, int layer, const void
     for (int i = 0; i < n_caches; ++i) {
         const svlm_cache* c = caches[i];
         if (!c) return SVLM_ERR_ARG;
-        if (c->dev.layers != c0->dev.layers || c->dev.kv_heads != c0->dev.kv_heads ||
-            c->dev.head_dim != c0->dev.head_dim || c->dev.n_slots != c0->dev.n_slots ||
-            c->dev.rope_mode != c0->dev.rope_mode || c->dev.sec_t != c0->dev.sec_t || c->dev.sec_th != c0->dev.sec_th ||
-            c->dev.theta[1] != c0->dev.theta[1] || c->device != c0->device)
-            return SVLM_ERR_ARG;
+        if (!same_geometry(c, c0)) return SVLM_ERR_ARG;
         if (n_q > c->appended) return SVLM_ERR_ORDER;
         fill_view(c, b.view[i]);
     }
@@ -160,9 +184,21 @@ int attend_common(svlm_cache* const* caches, int n_caches, int layer, const void
     const int n_layers = layer < 0 ? c0->dev.layers : 1;
     const int group = q_heads / c0->dev.kv_heads;
     int early = 0;
-    if (n_caches == 1 && n_q == 1 && layer >= 0) {
-        early = c0->last_decode_layer >= 0 && c0->last_decode_layer != layer;
-        c0->last_decode_layer = layer;
+    if (n_q == 1 && layer >= 0) {
+        // early loads: the kernel directly before this one on the stream was a decode of another layer that
+        // covered exactly these caches (it wrote neither their metadata nor this layer's pages)
+        early = 1;
+        for (int i = 0; i < n_caches; ++i) {
+            svlm_cache* c = caches[i];
+            if (c->last_decode_layer < 0 || c->last_decode_layer == layer || c->last_decode_batch != n_caches ||
+                c->last_decode_first != c0 || c->stream != c0->stream)
+                early = 0;
+        }
+        for (int i = 0; i < n_caches; ++i) {
+            caches[i]->last_decode_layer = layer;
+            caches[i]->last_decode_batch = n_caches;
+            caches[i]->last_decode_first = c0;
+        }
     } else {
         for (int i = 0; i < n_caches; ++i) caches[i]->last_decode_layer = -1;
     }
@@ -242,8 +278,10 @@ int svlm_cache_create(svlm_cache** out, int layers, int kv_heads, int head_dim, 
         d.tmaps = tm;
     }
     A(dev_alloc(c, &d.rope_tab, (size_t)3 * 256 * (head_dim / 2) * 2, false));
+    A(dev_alloc(c, &c->dev_copy, 1));
     if (rc == SVLM_OK) rc = make_tensor_maps(c);
     if (rc == SVLM_OK) rc = upload_rope_table(c);
+    if (rc == SVLM_OK) rc = sync_dev_copy(c);
     if (rc == SVLM_OK) {
         // pool pages on the free stack (top of the stack = lowest page number)
         std::vector<int> stack;
@@ -292,7 +330,8 @@ int svlm_cache_set_rope(svlm_cache* c, int mode, double base, const int sections
     c->dev.rope_mode = mode;
     fill_theta(c->dev, base);
     DeviceGuard guard(c->device);
-    return upload_rope_table(c);
+    const int rc = upload_rope_table(c);
+    return rc != SVLM_OK ? rc : sync_dev_copy(c);
 }
 
 int svlm_cache_set_policy(svlm_cache* c, int sink_any_type, int contiguous) {
@@ -300,7 +339,8 @@ int svlm_cache_set_policy(svlm_cache* c, int sink_any_type, int contiguous) {
     if (c->configured_locked) return SVLM_ERR_ORDER;
     c->dev.sink_any = sink_any_type ? 1 : 0;
     c->dev.contiguous = contiguous ? 1 : 0;
-    return SVLM_OK;
+    DeviceGuard guard(c->device);
+    return sync_dev_copy(c);
 }
 
 int svlm_cache_set_stream(svlm_cache* c, void* cuda_stream) {
@@ -339,6 +379,23 @@ int svlm_cache_evict(svlm_cache* c) {
     return SVLM_OK;
 }
 
+int svlm_cache_evict_batched(svlm_cache* const* caches, int n_caches) {
+    SvlmCacheList list;
+    const int rc = make_list(caches, n_caches, list);
+    if (rc != SVLM_OK) return rc;
+    svlm_cache* c0 = caches[0];
+    DeviceGuard guard(c0->device);
+    bool rotate = false;
+    for (int i = 0; i < n_caches; ++i) {
+        caches[i]->last_decode_layer = -1;
+        rotate = rotate || caches[i]->dev.contiguous;   // a cache with native positions never sets evict_moved
+    }
+    svlm_launch_evict_meta_batch(list, c0->stream);
+    if (rotate) svlm_launch_evict_rotate_batch(list, c0->dev, c0->stream);
+    SVLM_CUDA(cudaGetLastError());
+    return SVLM_OK;
+}
+
 int svlm_attend(svlm_cache* c, int layer, const void* Q, const int32_t* q_pos, int n_q, int q_heads, void* out) {
     if (!c) return SVLM_ERR_ARG;
     svlm_cache* one[1] = {c};
@@ -362,6 +419,32 @@ int svlm_decode_step(svlm_cache* c, int layer, const void* K, const void* V, con
     }
     svlm_cache* one[1] = {c};
     return attend_common(one, 1, layer, Q, pos, 1, q_heads, out, K, V);
+}
+
+int svlm_decode_step_batched(svlm_cache* const* caches, int n_caches, int layer, const void* K, const void* V,
+                             const uint8_t* token_type, const int32_t* pos, const void* Q, int q_heads, void* out) {
+    SvlmCacheList list;
+    const int rc = make_list(caches, n_caches, list);
+    if (rc != SVLM_OK) return rc;
+    svlm_cache* c0 = caches[0];
+    if (!K || !V || !pos || !Q || !out || layer < 0 || layer >= c0->dev.layers || q_heads < 1) return SVLM_ERR_ARG;
+    if (q_heads % c0->dev.kv_heads || q_heads / c0->dev.kv_heads > 8) return SVLM_ERR_ARG;
+    DeviceGuard guard(c0->device);
+    if (layer == 0) {
+        if (!token_type) return SVLM_ERR_ARG;
+        for (int i = 0; i < n_caches; ++i) {
+            svlm_cache* c = caches[i];
+            c->configured_locked = true;
+            c->last_decode_layer = -1;
+            c->appended += 1;
+            c->pending_n = 1;
+        }
+        svlm_launch_append_meta_batch(list, token_type, pos, 1, c0->stream);
+    } else {
+        for (int i = 0; i < n_caches; ++i)
+            if (caches[i]->pending_n != 1) return SVLM_ERR_ORDER;
+    }
+    return attend_common(caches, n_caches, layer, Q, pos, 1, q_heads, out, K, V);
 }
 
 int svlm_attend_batched(svlm_cache* const* caches, int n_caches, int layer, const void* Q, const int32_t* q_pos,

@@ -145,35 +145,40 @@ def test_config3_full_stack_steady_state_step_as_benchmarked():
 
 
 def test_config4_batched_decode_16_streams_with_interleaved_eviction():
-    """16 independent streams at the full retained size, 48 batched q=1 steps (one launch for all streams), an
+    """16 independent streams at the full retained size, 48 batched q=1 steps (svlm_decode_step_batched), a batched
     eviction every 16 steps; every stream's output compared at sampled steps, metadata after every eviction."""
     from harness import bits_to_dev, dev_to_f64
     from paper_2510_09608_b200 import binding, streamgen as sg
     wl = dataclasses.replace(sg.workloads()[4], decode_steps=16)
-    sides = []
+    sides, fill_evicts = [], []
     for sid in range(wl.streams):
         stream, cache, ref = _setup(wl, sid)
-        _fill(cache, ref, wl, stream)
+        fill_evicts.append(_fill(cache, ref, wl, stream))
         _give(ref, stream, 0)
         sides.append((stream, cache, ref))
+    caches = [c for _, c, _ in sides]
     for step in range(48):
         toks = [s.next_decode_token() for s, _, _ in sides]
         for (s, c, r), (g1, t1, p1) in zip(sides, toks):
-            c.append(0, bits_to_dev(s.k(0, g1)), bits_to_dev(s.v(0, g1)), torch.from_numpy(t1).cuda(),
-                     torch.from_numpy(np.ascontiguousarray(p1)).cuda())
             r.append(None, None, t1, p1)
             _give_new(r, s, 0, g1)
+        gen = lambda f: bits_to_dev(np.stack([f(s, g1)[0] for (s, _, _), (g1, _, _) in zip(sides, toks)]))  # noqa: E731
         Q = np.stack([s.q(0, g1) for (s, _, _), (g1, _, _) in zip(sides, toks)])
-        qpos = torch.from_numpy(np.stack([p1 for _, _, p1 in toks])).cuda()
-        out = dev_to_f64(binding.attend_batched([c for _, c, _ in sides], 0, bits_to_dev(Q), qpos))
+        ty = torch.from_numpy(np.concatenate([t1 for _, t1, _ in toks])).cuda()
+        qpos = torch.from_numpy(np.ascontiguousarray(np.stack([p1[0] for _, _, p1 in toks]))).cuda()
+        # as benchmarked: one fused step for all streams (metadata launch + attention launch)
+        out = dev_to_f64(binding.decode_step_batched(caches, 0, gen(lambda s, g: s.k(0, g)), gen(lambda s, g: s.v(0, g)), ty,
+                                                     qpos, bits_to_dev(Q[:, 0])))
         if step % 16 in (0, 15):
             for i, ((s, c, r), (g1, t1, p1)) in enumerate(zip(sides, toks)):
-                _close(out[i], r.attend(0, Q[i], p1), f"stream {i} step {step}")
+                _close(out[i][None], r.attend(0, Q[i], p1), f"stream {i} step {step}")
         if step % 16 == 15:
+            binding.evict_batched(caches)
             for s, c, r in sides:
-                c.evict()
                 r.evict()
                 _same_metadata(c, r)
+    for (s, c, r), n_ev in list(zip(sides, fill_evicts))[::5]:
+        _check_kv(c, r, s, wl, 0, n_ev + 3)
 
 
 def test_config5_high_frame_rate_streams_sampled():

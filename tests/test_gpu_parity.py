@@ -148,6 +148,55 @@ def test_batched_streams_match_single_calls():
         assert err.max() <= 1e-2 and err.mean() <= 1e-3
 
 
+@pytest.mark.parametrize("rope_1d", [False, True])
+def test_batched_decode_steps_and_batched_evict(rope_1d):
+    """Three streams at different fill levels advance in lock step through svlm_decode_step_batched (two layers,
+    one launch per layer for all streams) with svlm_cache_evict_batched every four tokens: outputs of every
+    stream, layer and step against the checker, metadata bit-exact after every eviction, stored K/V at the end."""
+    from harness import SideBySide, assert_close, bits_to_dev, dev_to_f64
+    from paper_2510_09608_b200 import binding
+    wl = dataclasses.replace(_wl(2), layers=2, n_sink=16, vision_window=256, text_window=24, frames=1, grid_h=8, grid_w=8)
+    if rope_1d:
+        wl = dataclasses.replace(_wl(1), layers=2, q_heads=8, kv_heads=2)
+    sides = [SideBySide(wl, stream=i) for i in range(3)]
+    for i, s in enumerate(sides):
+        for _ in range(3 + 2 * i):
+            s.append_chunk()
+            s.evict()
+    caches = [s.cache for s in sides]
+    for step in range(10):
+        toks = [s.stream.next_decode_token() for s in sides]
+        ty = torch.from_numpy(np.concatenate([t[1] for t in toks])).cuda()
+        ps = torch.from_numpy(np.ascontiguousarray(np.stack([t[2][0] for t in toks]))).cuda()
+        outs, Qs = [], []
+        for l in range(wl.layers):
+            K = np.stack([s.stream.k(l, t[0])[0] for s, t in zip(sides, toks)])
+            V = np.stack([s.stream.v(l, t[0])[0] for s, t in zip(sides, toks)])
+            Qs.append(np.stack([s.stream.q(l, t[0])[0] for s, t in zip(sides, toks)]))
+            outs.append(dev_to_f64(binding.decode_step_batched(caches, l, bits_to_dev(K), bits_to_dev(V),
+                                                               ty if l == 0 else None, ps, bits_to_dev(Qs[-1]))))
+        for i, (s, t) in enumerate(zip(sides, toks)):
+            assert s.cache.status() == binding.OK
+            s.ref.append(None, None, t[1], t[2])
+            s.last = t
+            for l in range(wl.layers):
+                s._give_values_to_ref(l)
+                assert_close(s._stats(outs[l][i][None], s.ref.attend(l, Qs[l][i][None], t[2])))
+        if step % 4 == 3:
+            binding.evict_batched(caches)
+            for s in sides:
+                s.ref.evict()
+                s.n_evicts += 1
+                s.check_metadata()
+    for s in sides:
+        s.check_metadata()
+        for l in range(wl.layers):
+            s.check_kv(l)
+    with pytest.raises(binding.SvlmError) as e:          # a cache may appear only once in a batch
+        binding.evict_batched([caches[0], caches[0]])
+    assert e.value.status == binding.ERR_ARG
+
+
 def test_errors_and_capacity():
     from paper_2510_09608_b200 import binding
     with pytest.raises(binding.SvlmError):
