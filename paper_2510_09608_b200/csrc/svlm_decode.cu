@@ -518,9 +518,11 @@ size_t svlm_decode_ws_floats(int layers, int kv_heads, int head_dim, int splits)
 }
 
 int svlm_decode_splits(int n_pages, int kv_heads, int problems) {
-    // one CTA per SM: the combine reads every split's partial once, so more splits than needed to
-    // fill the machine only lengthen the tail
-    int splits = 148 / (kv_heads * problems);
+    // One problem (a single stream's layer): one CTA per SM, since the combine reads every split's
+    // partial once and more splits than needed to fill the machine only lengthen the tail.  Several
+    // problems in one launch: up to two resident CTAs per SM (measured on 16 streams x 4 KV heads:
+    // 256 CTAs 64 us, 128 CTAs 70 us, 384 CTAs, which no longer fit at once, 74 us).
+    int splits = (problems > 1 ? 296 : 148) / (kv_heads * problems);
     splits = splits < 1 ? 1 : splits;
     return splits > 4 * n_pages ? 4 * n_pages : splits;
 }

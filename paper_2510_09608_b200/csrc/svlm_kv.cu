@@ -28,16 +28,42 @@ __device__ __forceinline__ void rotate8(Bf16x8& lo, Bf16x8& hi, const float* cs,
     }
 }
 
-// One thread per (token, group of 8 pairs); it serves every kv head (and every layer when
-// layer < 0) of that token, so the rotation factors are looked up once (table, see svlm_rope.cuh).
+// One thread per (token, group of 8 pairs); it serves the kv heads of its share of the layers
+// (grid.y splits the layers when layer < 0), so the rotation factors are looked up once (table, see
+// svlm_rope.cuh).  The source rows do not depend on the metadata, so the loads of the first rows are
+// issued before the chain slot -> position -> factors is walked.
+template <int UNROLL>
 __global__ void __launch_bounds__(256) kv_write_kernel(SvlmCacheDev cd, int layer, const uint16_t* __restrict__ K,
-                                                       const uint16_t* __restrict__ V, int n) {
-    if (cd.ctrl->append_n != n) return;   // the metadata append was dropped (capacity) or does not match
+                                                       const uint16_t* __restrict__ V, int n, int layers_per_block) {
     const int half = cd.head_dim / 2;
     const int groups = half / 8;          // threads per token
     const int t = blockIdx.x * blockDim.x + threadIdx.x;
     const int i = t / groups, g = t % groups;
     if (i >= n) return;
+    const int d = cd.head_dim;
+    const int l0 = layer < 0 ? blockIdx.y * layers_per_block : layer;
+    const int l1 = layer < 0 ? min(cd.layers, l0 + layers_per_block) : layer + 1;
+    const int row0 = l0 * cd.kv_heads, row1 = l1 * cd.kv_heads;      // rows of [layer][kv_head]
+    // source of row r: [layer (only when all layers are given)][token][kv_head]
+    auto src_of = [&](int r) {
+        const int l = r / cd.kv_heads, h = r % cd.kv_heads;
+        return (((size_t)(layer < 0 ? l : 0) * n + i) * cd.kv_heads + h) * d + g * 8;
+    };
+    Bf16x8 lo[UNROLL], hi[UNROLL];
+    uint4 vlo[UNROLL], vhi[UNROLL];
+    auto load_rows = [&](int r) {
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u)
+            if (r + u < row1) {
+                const size_t src = src_of(r + u);
+                lo[u] = *reinterpret_cast<const Bf16x8*>(K + src);
+                hi[u] = *reinterpret_cast<const Bf16x8*>(K + src + half);
+                vlo[u] = *reinterpret_cast<const uint4*>(V + src);
+                vhi[u] = *reinterpret_cast<const uint4*>(V + src + half);
+            }
+    };
+    load_rows(row0);
+    if (cd.ctrl->append_n != n) return;   // the metadata append was dropped (capacity) or does not match
     const int slot = cd.new_slot[i];
     // A layer's keys may arrive after an eviction has already shifted these tokens (layers are
     // computed one after another): rotate at the slot's CURRENT position, and skip a token that
@@ -53,22 +79,18 @@ __global__ void __launch_bounds__(256) kv_write_kernel(SvlmCacheDev cd, int laye
         cs[j] = f.x;
         sn[j] = f.y;
     }
-    const int d = cd.head_dim;
-    const int l0 = layer < 0 ? 0 : layer, l1 = layer < 0 ? cd.layers : layer + 1;
-    for (int l = l0; l < l1; ++l) {
-        for (int h = 0; h < cd.kv_heads; ++h) {
-            const size_t src = (((size_t)(layer < 0 ? l : 0) * n + i) * cd.kv_heads + h) * d;
-            const size_t dst = (((size_t)l * cd.kv_heads + h) * cd.n_slots + slot) * d;
-            Bf16x8 lo = *reinterpret_cast<const Bf16x8*>(K + src + g * 8);
-            Bf16x8 hi = *reinterpret_cast<const Bf16x8*>(K + src + half + g * 8);
-            const uint4 vlo = *reinterpret_cast<const uint4*>(V + src + g * 8);
-            const uint4 vhi = *reinterpret_cast<const uint4*>(V + src + half + g * 8);
-            rotate8(lo, hi, cs, sn);
-            *reinterpret_cast<Bf16x8*>(cd.K + dst + g * 8) = lo;
-            *reinterpret_cast<Bf16x8*>(cd.K + dst + half + g * 8) = hi;
-            *reinterpret_cast<uint4*>(cd.V + dst + g * 8) = vlo;
-            *reinterpret_cast<uint4*>(cd.V + dst + half + g * 8) = vhi;
-        }
+    for (int r = row0; r < row1; r += UNROLL) {
+        if (r != row0) load_rows(r);
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u)
+            if (r + u < row1) {
+                const size_t dst = ((size_t)(r + u) * cd.n_slots + slot) * d + g * 8;
+                rotate8(lo[u], hi[u], cs, sn);
+                *reinterpret_cast<Bf16x8*>(cd.K + dst) = lo[u];
+                *reinterpret_cast<Bf16x8*>(cd.K + dst + half) = hi[u];
+                *reinterpret_cast<uint4*>(cd.V + dst) = vlo[u];
+                *reinterpret_cast<uint4*>(cd.V + dst + half) = vhi[u];
+            }
     }
 }
 
@@ -142,7 +164,9 @@ int rotate_layers_per_block(int layers, int kv_heads) {
 void svlm_launch_kv_write(const SvlmCacheDev& cd, int layer, const void* K, const void* V, int n, cudaStream_t st) {
     const int groups = cd.head_dim / 16;
     const int threads = n * groups;
-    kv_write_kernel<<<(threads + 255) / 256, 256, 0, st>>>(cd, layer, (const uint16_t*)K, (const uint16_t*)V, n);
+    const int lpb = rotate_layers_per_block(cd.layers, cd.kv_heads);
+    dim3 grid((threads + 255) / 256, layer < 0 ? (cd.layers + lpb - 1) / lpb : 1);
+    kv_write_kernel<4><<<grid, 256, 0, st>>>(cd, layer, (const uint16_t*)K, (const uint16_t*)V, n, lpb);
     svlm_count_launch();
 }
 

@@ -278,12 +278,21 @@ __device__ __forceinline__ int count_below(const long long* g, int n, long long 
     return lo;
 }
 
+constexpr int EV_SMEM = 2048;   // evicted tokens of one call whose lists also fit in shared memory
+constexpr int KEPT_BATCH = 5;   // retained tokens a thread handles per round (loads of a round are issued together)
+
 // ---------------------------------------------------------------------------------------------
 // Evict: keep-mask (a suffix of each ring plus the sinks), prefix sums of the evicted tokens'
 // cursor advances, and the left-shift E(i) of every retained token i: the advances of all evicted
 // tokens that precede it in the stream.
+//
+// The kernel is a chain of dependent round trips to L2 (page table -> slot -> ordinal -> search ->
+// position), so every stage issues the loads of all its items before it uses any of them, and the
+// lists that the searches walk sit in shared memory when they fit.
 __device__ __forceinline__ void evict_meta_body(const SvlmCacheDev& cd) {
-    __shared__ long long wbuf64[META_WARPS];
+    __shared__ long long wbuf64[2][META_WARPS];
+    __shared__ long long s_gid[EV_SMEM];       // ordinals of the evicted tokens: text ring, then vision ring
+    __shared__ long long s_pref[EV_SMEM + 2];  // exclusive prefix sums of their advances (n+1 entries per ring)
     __shared__ int s_moved;
     SvlmCtrl* ctrl = cd.ctrl;
     const int tid = threadIdx.x;
@@ -292,6 +301,7 @@ __device__ __forceinline__ void evict_meta_body(const SvlmCacheDev& cd) {
     const long long ring_n[2] = {ctrl->ring_n[0], ctrl->ring_n[1]};
     const long long lo0[2] = {ctrl->ring_lo[0], ctrl->ring_lo[1]};
     const int sink_fill = ctrl->sink_fill;
+    const int free_top0 = ctrl->free_top;
     const int win[2] = {cd.text_window, cd.vision_window};
     long long lo1[2];
     int n_ev[2];
@@ -299,63 +309,107 @@ __device__ __forceinline__ void evict_meta_body(const SvlmCacheDev& cd) {
         lo1[t] = min(ring_n[t], max(lo0[t], ring_n[t] - (long long)win[t]));
         n_ev[t] = (int)(lo1[t] - lo0[t]);
     }
+    const bool in_smem = n_ev[0] + n_ev[1] <= EV_SMEM;
+    // where the searches read the lists of ring t
+    const long long* gid_list[2] = {in_smem ? s_gid : cd.ev_gid[0], in_smem ? s_gid + n_ev[0] : cd.ev_gid[1]};
+    const long long* pref_list[2] = {in_smem ? s_pref : cd.ev_pref[0], in_smem ? s_pref + n_ev[0] + 1 : cd.ev_pref[1]};
     __syncthreads();
 
-    // evicted tokens of each ring in ordinal (= stream) order, with exclusive prefix sums of a
-    long long freed[2];
-    for (int t = 0; t < 2; ++t) {
-        long long carry = 0;
-        for (int base = 0; base < n_ev[t]; base += META_THREADS) {
-            const int i = base + tid;
-            long long a = 0;
-            int slot = -1;
-            if (i < n_ev[t]) {
-                slot = ring_slot(cd, t, lo0[t] + i);
-                a = cd.contiguous ? cd.slot_a[slot] : 0;
-                cd.ev_gid[t][i] = cd.slot_gid[slot];
+    // evicted tokens of both rings in ordinal (= stream) order, with exclusive prefix sums of a
+    long long freed[2] = {0, 0};
+    for (int base = 0; base < max(n_ev[0], n_ev[1]); base += META_THREADS) {
+        const int i = base + tid;
+        int slot[2] = {-1, -1};
+        long long a[2] = {0, 0}, g[2] = {0, 0};
+#pragma unroll
+        for (int t = 0; t < 2; ++t)
+            if (i < n_ev[t]) slot[t] = ring_slot(cd, t, lo0[t] + i);
+#pragma unroll
+        for (int t = 0; t < 2; ++t)
+            if (slot[t] >= 0) {
+                a[t] = cd.contiguous ? cd.slot_a[slot[t]] : 0;
+                g[t] = cd.slot_gid[slot[t]];
             }
-            const long long ex = block_excl_sum64(a, carry, wbuf64);
-            if (i < n_ev[t]) {
-                cd.ev_pref[t][i] = ex;
-                cd.slot_gid[slot] = -1;
-                cd.slot_delta[slot] = 0;
+#pragma unroll
+        for (int t = 0; t < 2; ++t) {
+            if (base >= n_ev[t]) continue;            // uniform over the block
+            const long long ex = block_excl_sum64(a[t], freed[t], wbuf64[t]);
+            if (slot[t] >= 0) {
+                if (in_smem) {
+                    s_gid[(t ? n_ev[0] : 0) + i] = g[t];
+                    s_pref[(t ? n_ev[0] + 1 : 0) + i] = ex;
+                } else {
+                    cd.ev_gid[t][i] = g[t];
+                    cd.ev_pref[t][i] = ex;
+                }
+                cd.slot_gid[slot[t]] = -1;
+                cd.slot_delta[slot[t]] = 0;
             }
         }
-        freed[t] = carry;
-        if (tid == 0) cd.ev_pref[t][n_ev[t]] = carry;
     }
+    if (tid == 0)
+        for (int t = 0; t < 2; ++t) {
+            if (in_smem) s_pref[(t ? n_ev[0] + 1 : 0) + n_ev[t]] = freed[t];
+            else cd.ev_pref[t][n_ev[t]] = freed[t];
+        }
     __syncthreads();
 
     // retained tokens: sinks, then the kept suffix of each ring
     const long long kept_ring[2] = {ring_n[0] - lo1[0], ring_n[1] - lo1[1]};
     const long long n_kept = sink_fill + kept_ring[0] + kept_ring[1];
     int moved = 0;
-    for (long long i = tid; i < n_kept; i += META_THREADS) {
-        int slot;
-        if (i < sink_fill) slot = (int)i;
-        else if (i < sink_fill + kept_ring[0]) slot = ring_slot(cd, 0, lo1[0] + (i - sink_fill));
-        else slot = ring_slot(cd, 1, lo1[1] + (i - sink_fill - kept_ring[0]));
-        const long long g = cd.slot_gid[slot];
-        long long E = 0;
-        for (int t = 0; t < 2; ++t)
-            if (n_ev[t]) E += cd.ev_pref[t][count_below(cd.ev_gid[t], n_ev[t], g)];
-        cd.slot_delta[slot] = (int)E;
-        if (E) {
-            moved = 1;
-            for (int k = 0; k < 3; ++k) cd.slot_c[k * cd.n_slots + slot] -= (int)E;
+    for (long long base = 0; base < n_kept; base += (long long)KEPT_BATCH * META_THREADS) {
+        int slot[KEPT_BATCH];
+        long long g[KEPT_BATCH];
+        int E[KEPT_BATCH], c[KEPT_BATCH][3];
+#pragma unroll
+        for (int u = 0; u < KEPT_BATCH; ++u) {
+            const long long i = base + (long long)u * META_THREADS + tid;
+            if (i >= n_kept) slot[u] = -1;
+            else if (i < sink_fill) slot[u] = (int)i;
+            else if (i < sink_fill + kept_ring[0]) slot[u] = ring_slot(cd, 0, lo1[0] + (i - sink_fill));
+            else slot[u] = ring_slot(cd, 1, lo1[1] + (i - sink_fill - kept_ring[0]));
+        }
+#pragma unroll
+        for (int u = 0; u < KEPT_BATCH; ++u) {
+            g[u] = slot[u] >= 0 ? cd.slot_gid[slot[u]] : 0;
+#pragma unroll
+            for (int k = 0; k < 3; ++k) c[u][k] = slot[u] >= 0 ? cd.slot_c[k * cd.n_slots + slot[u]] : 0;
+        }
+#pragma unroll
+        for (int u = 0; u < KEPT_BATCH; ++u) {
+            long long e = 0;
+            if (slot[u] >= 0)
+                for (int t = 0; t < 2; ++t)
+                    if (n_ev[t]) e += pref_list[t][count_below(gid_list[t], n_ev[t], g[u])];
+            E[u] = (int)e;
+        }
+#pragma unroll
+        for (int u = 0; u < KEPT_BATCH; ++u) {
+            if (slot[u] < 0) continue;
+            cd.slot_delta[slot[u]] = E[u];
+            if (E[u]) {
+                moved = 1;
+#pragma unroll
+                for (int k = 0; k < 3; ++k) cd.slot_c[k * cd.n_slots + slot[u]] = c[u][k] - E[u];
+            }
         }
     }
     if (moved) s_moved = 1;
 
-    // release pages that fell wholly below the new low-water mark
-    if (tid == 0) {
-        int top = ctrl->free_top;
+    // release the pages that fell wholly below the new low-water mark (text ring's first, in ring order)
+    {
+        long long first[2], cnt[2];
         for (int t = 0; t < 2; ++t) {
-            const long long end = min(lo1[t] / SVLM_PAGE, ceil_page(ring_n[t]));
-            for (long long k = lo0[t] / SVLM_PAGE; k < end; ++k)
-                cd.free_stack[top++] = cd.page_table[t][(int)k & (cd.pt_size - 1)];
+            first[t] = lo0[t] / SVLM_PAGE;
+            cnt[t] = max(0ll, min(lo1[t] / SVLM_PAGE, ceil_page(ring_n[t])) - first[t]);
         }
-        ctrl->free_top = top;
+        for (long long i = tid; i < cnt[0] + cnt[1]; i += META_THREADS) {
+            const int t = i < cnt[0] ? 0 : 1;
+            const long long k = first[t] + (t ? i - cnt[0] : i);
+            cd.free_stack[free_top0 + i] = cd.page_table[t][(int)k & (cd.pt_size - 1)];
+        }
+        if (tid == 0) ctrl->free_top = free_top0 + (int)(cnt[0] + cnt[1]);
     }
     __syncthreads();
     rebuild_tiles(cd, sink_fill, lo1, ring_n);
