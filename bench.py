@@ -166,6 +166,55 @@ def run_step(cache, wl, inp, timers=None):
         timed("decode_token", lambda: decode_token(d))
 
 
+def stack_decode_inputs(inps):
+    """Per generated token, the streams' one-token inputs side by side: K, V, Q as [layers][streams][heads][d],
+    types [streams], pos [streams](x3), the layout of svlm_decode_step_batched."""
+    import torch
+    toks = []
+    for t in range(len(inps[0].dec)):
+        d = {k: torch.stack([inp.dec[t][k][:, 0] for inp in inps], dim=1).contiguous() for k in ("K", "V", "Q")}
+        d["types"] = torch.cat([inp.dec[t]["types"] for inp in inps]).contiguous()
+        d["pos"] = torch.stack([inp.dec[t]["pos"][0] for inp in inps]).contiguous()
+        d["out"] = torch.empty_like(d["Q"])
+        toks.append(d)
+    return toks
+
+
+def run_step_multi(caches, wl, inps, dec, timers=None):
+    """One step of several streams that advance in lock step: every stream appends its chunk, ONE batched
+    eviction, chunk prefill per stream and layer (the chunks differ in length), then the generated tokens with one
+    batched decode launch per layer for all streams.  inps: one StepInputs per stream; dec: stack_decode_inputs."""
+    import torch
+    from paper_2510_09608_b200 import binding
+    L = wl.layers
+
+    def timed(name, fn):
+        if timers is None:
+            return fn()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        fn()
+        b.record()
+        timers.setdefault(name, []).append((a, b))
+
+    for c, inp in zip(caches, inps):
+        timed("append", lambda: c.append(0, inp.K[0], inp.V[0], inp.types, inp.pos))
+    timed("evict", lambda: binding.evict_batched(caches))
+    for l in range(L):
+        for c, inp in zip(caches, inps):
+            if l:
+                timed("append", lambda: c.append(l, inp.K[l], inp.V[l]))
+            timed("prefill", lambda: c.attend(l, inp.Q[l], inp.pos, inp.out[l]))
+
+    def decode_token(d):
+        for l in range(L):
+            binding.decode_step_batched(caches, l, d["K"][l], d["V"][l], d["types"] if l == 0 else None, d["pos"],
+                                        d["Q"][l], d["out"][l])
+
+    for d in dec:
+        timed("decode_token", lambda: decode_token(d))
+
+
 def run_step_host(cache, wl, inp):
     """The same step through the host-buffer entry points (all layers per call): copies included."""
     cache.append_host(-1, inp.h["K"], inp.h["V"], inp.h["types"], inp.h["pos"])
@@ -369,6 +418,120 @@ def bench_batched_decode(args, wl, base, peaks, rank, world, local):
                               steps=timed_cycles * cycle)))
 
 
+def bench_multi_stream(args, wl, base, config, peaks, rank, world, local):
+    """Workload 5: `wl.streams` streams of a full attention stack in lock step; a step is one chunk of every stream
+    (append, batched eviction, per-stream chunk prefill, batched decode).  Steps are replayed from CUDA graphs;
+    value = frames/s over all streams."""
+    import torch
+    from paper_2510_09608_b200 import binding
+    S = wl.streams
+    streams = [sg.Stream(wl, rank * S + i) for i in range(S)]
+    caches = []
+    fill_chunks = 0
+    for st in streams:
+        c = binding.Cache(wl.layers, wl.kv_heads, wl.head_dim, wl.n_sink, wl.vision_window, wl.text_window, wl.capacity)
+        c.set_rope(wl.rope_mode, wl.rope_base, wl.sections)
+        fill_chunks = fill_to_steady_state(c, wl, st)
+        c.evict()
+        assert c.status() == binding.OK
+        caches.append(c)
+
+    def make_step():
+        inps = [StepInputs(wl, st, *next_step_schedule(st, wl)) for st in streams]
+        return inps, stack_decode_inputs(inps)
+
+    total = args.warmup + args.steps
+    steps = [make_step() for _ in range(total)]
+    prime = make_step()
+    # one plain step on scratch caches: one-time function attributes are set outside any capture
+    scratch = []
+    for _ in range(S):
+        c = binding.Cache(wl.layers, wl.kv_heads, wl.head_dim, wl.n_sink, wl.vision_window, wl.text_window, wl.capacity)
+        c.set_rope(wl.rope_mode, wl.rope_base, wl.sections)
+        scratch.append(c)
+    run_step_multi(scratch, wl, *steps[0])
+    torch.cuda.synchronize()
+    for c in scratch:
+        c.close()
+
+    graphs, launches = [], []
+    cur = torch.cuda.current_stream()
+    for inps, dec in steps:
+        g = torch.cuda.CUDAGraph()
+        before = binding.launch_count()
+        with torch.cuda.graph(g):
+            for c in caches:
+                c.set_stream(torch.cuda.current_stream())
+            run_step_multi(caches, wl, inps, dec)
+        launches.append(binding.launch_count() - before)
+        graphs.append(g)
+    for c in caches:
+        c.set_stream(cur)
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(args.warmup):
+        graphs[i].replay()
+    sampler = ClockSampler(local)
+    barrier()
+    sampler.start()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    ev[0].record()
+    for i in range(args.steps):
+        graphs[args.warmup + i].replay()
+        ev[i + 1].record()
+    barrier()
+    clocks = sampler.finish()
+    step_ms = [ev[i].elapsed_time(ev[i + 1]) for i in range(args.steps)]
+    ms_per_step = max_over_ranks(ev[0].elapsed_time(ev[-1]), world) / args.steps
+    for c in caches:
+        assert c.status() == binding.OK
+
+    # per-kernel durations: one plain pass with events around every call
+    timers = {}
+    run_step_multi(caches, wl, *prime, timers)
+    torch.cuda.synchronize()
+    kern = {k: [a.elapsed_time(b) for a, b in v] for k, v in timers.items()}
+    avg = {k: statistics.mean(v) for k, v in kern.items()}
+    tot = {k: sum(v) for k, v in kern.items()}
+    n_q = statistics.mean(inp.n for inp in prime[0])
+    lk = wl.retained
+    flops = prefill_flops(wl, int(round(n_q)), lk)
+    kv_bytes_layer = lk * 2 * wl.kv_heads * wl.head_dim * 2 * S          # one batched decode launch: all streams, one layer
+    evict_bytes = 2 * (wl.retained - wl.n_sink) * wl.kv_heads * wl.head_dim * 2 * wl.layers * S
+    kernels = {
+        "prefill": dict(bound="tensor", avg_ms=avg["prefill"], per_step_ms=tot["prefill"],
+                        achieved=flops / (avg["prefill"] * 1e-3) / 1e12, unit="TFLOP/s", peak=peaks["bf16_burst"]),
+        "decode": dict(bound="hbm", avg_ms=avg["decode_token"] / wl.layers, per_step_ms=tot["decode_token"],
+                       achieved=kv_bytes_layer * wl.layers / (avg["decode_token"] * 1e-3) / 1e9, unit="GB/s",
+                       peak=peaks["hbm"], note="avg_ms = time of one token step of all streams over all layers / layers"),
+        "evict": dict(bound="hbm", avg_ms=avg["evict"], per_step_ms=tot["evict"],
+                      achieved=evict_bytes / (avg["evict"] * 1e-3) / 1e9, unit="GB/s", peak=peaks["hbm"]),
+        "append": dict(avg_ms=avg["append"], per_step_ms=tot["append"]),
+    }
+    for k in ("prefill", "decode", "evict"):
+        kernels[k]["frac"] = kernels[k]["achieved"] / kernels[k]["peak"]
+    dominant = max(("prefill", "decode", "evict"), key=lambda k: kernels[k]["per_step_ms"])
+    kd = kernels[dominant]
+    roofline = dict(bound="tensor" if dominant == "prefill" else "hbm", kernel=dominant, achieved=kd["achieved"],
+                    peak=kd["peak"], unit=kd["unit"], frac=kd["frac"], traffic=None,
+                    algorithmic=(flops if dominant == "prefill" else kv_bytes_layer if dominant == "decode" else evict_bytes),
+                    peak_source=peaks["source"] + (" (burst bf16)" if dominant == "prefill" else " (copy)"))
+    if rank == 0:
+        config = dict(config, replicas="independent streams, no collective",
+                      streams=f"{S} streams per GPU in lock step: batched eviction and decode, per-stream prefill")
+        print(json.dumps(dict(base, value=whole_job_value(world, wl.frames * S, ms_per_step), ms_per_step=ms_per_step,
+                              config=config, roofline=roofline, cpu_baseline=None, e2e=None,
+                              gpu_launches=int(sum(launches[args.warmup:])), clocks=clocks, kernels=kernels,
+                              decode_tok_s=wl.decode_steps * S / (tot["decode_token"] * 1e-3),
+                              step_ms=dict(min=min(step_ms), median=statistics.median(step_ms), max=max(step_ms)),
+                              state=dict(fill_chunks=fill_chunks, cuda_graph=True))))
+
+
 def dataclasses_replace(obj, **kw):
     import dataclasses
     return dataclasses.replace(obj, **kw)
@@ -439,6 +602,11 @@ def main():
     peaks = load_peaks()
     if wl.streams > 1 and wl.layers == 1:
         bench_batched_decode(args, wl, base, peaks, rank, world, local)
+        if world > 1:
+            dist.destroy_process_group()
+        return
+    if wl.streams > 1:
+        bench_multi_stream(args, wl, base, config, peaks, rank, world, local)
         if world > 1:
             dist.destroy_process_group()
         return

@@ -182,37 +182,42 @@ def test_config4_batched_decode_16_streams_with_interleaved_eviction():
 
 
 def test_config5_high_frame_rate_streams_sampled():
-    """The 8 frames/s x 8x8-grid shape (vision blocks of span 8, text bursts up to 32): two of the eight streams,
-    four of the 28 layers, one steady-state step each, layer-sequential calls as benchmarked."""
+    """The 8 frames/s x 8x8-grid shape (vision blocks of span 8, text bursts up to 32): three of the eight streams,
+    four of the 28 layers, one steady-state step run as benchmarked: the streams advance in lock step (per-stream
+    appends and chunk prefill, one batched eviction, one batched decode launch per layer and token)."""
     import bench
     from harness import dev_to_f64
     from paper_2510_09608_b200 import streamgen as sg
     wl = dataclasses.replace(sg.workloads()[5], layers=4)
     rng = np.random.default_rng(wl.seed)
-    for sid in (0, 7):
+    sides, fills = [], []
+    for sid in (0, 3, 7):
         stream, cache, ref = _setup(wl, sid)
-        n_evicts = _fill(cache, ref, wl, stream)
+        fills.append(_fill(cache, ref, wl, stream))
         _same_metadata(cache, ref)
-        chunk, decode = bench.next_step_schedule(stream, wl)
-        inp = bench.StepInputs(wl, stream, chunk, decode)
-        bench.run_step(cache, wl, inp)
-        torch.cuda.synchronize()
+        sides.append((stream, cache, ref))
+    scheds = [bench.next_step_schedule(s, wl) for s, _, _ in sides]
+    inps = [bench.StepInputs(wl, s, chunk, decode) for (s, _, _), (chunk, decode) in zip(sides, scheds)]
+    dec = bench.stack_decode_inputs(inps)
+    bench.run_step_multi([c for _, c, _ in sides], wl, inps, dec)
+    torch.cuda.synchronize()
+    for i, ((stream, cache, ref), (chunk, decode), inp) in enumerate(zip(sides, scheds, inps)):
         gids, types, pos = chunk
         ref.append(None, None, types, pos)
         ref.evict()
         rows = np.unique(np.concatenate([[0, len(gids) - 1], rng.integers(0, len(gids), 16)]))
         for l in (0, 3):
             _give(ref, stream, l)
-            _close(dev_to_f64(inp.out[l])[rows], ref.attend(l, stream.q(l, gids), pos, rows), f"stream {sid} prefill layer {l}")
-        for d, (g1, t1, p1) in zip(inp.dec, decode):
+            _close(dev_to_f64(inp.out[l])[rows], ref.attend(l, stream.q(l, gids), pos, rows), f"stream {i} prefill layer {l}")
+        for g1, t1, p1 in decode:
             ref.append(None, None, t1, p1)
             for l in (0, 3):
                 _give_new(ref, stream, l, g1)
         for l in (0, 3):
             g1, t1, p1 = decode[-1]
-            _close(dev_to_f64(inp.dec[-1]["out"][l]), ref.attend(l, stream.q(l, g1), p1), f"stream {sid} last decode layer {l}")
+            _close(dev_to_f64(dec[-1]["out"][l][i])[None], ref.attend(l, stream.q(l, g1), p1), f"stream {i} last decode layer {l}")
         _same_metadata(cache, ref)
-        _check_kv(cache, ref, stream, wl, 3, n_evicts + 1)
+        _check_kv(cache, ref, stream, wl, 3, fills[i] + 1)
 
 
 def test_config2_whole_600_chunk_stream_metadata_and_final_outputs():
