@@ -279,7 +279,18 @@ __device__ __forceinline__ int count_below(const long long* g, int n, long long 
 }
 
 constexpr int EV_SMEM = 2048;   // evicted tokens of one call whose lists also fit in shared memory
-constexpr int KEPT_BATCH = 5;   // retained tokens a thread handles per round (loads of a round are issued together)
+constexpr int KEPT_BATCH = 2;   // retained tokens a thread handles per round (loads of a round are issued together)
+constexpr int EV_CLUSTER = 8;   // CTAs (one thread-block cluster) that share the retained tokens of one cache
+
+__device__ __forceinline__ unsigned cluster_ctarank() {
+    unsigned r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// All threads of all CTAs of the cluster; orders their global-memory accesses before and after it.
+__device__ __forceinline__ void cluster_barrier() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\nbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
 
 // ---------------------------------------------------------------------------------------------
 // Evict: keep-mask (a suffix of each ring plus the sinks), prefix sums of the evicted tokens'
@@ -288,8 +299,12 @@ constexpr int KEPT_BATCH = 5;   // retained tokens a thread handles per round (l
 //
 // The kernel is a chain of dependent round trips to L2 (page table -> slot -> ordinal -> search ->
 // position), so every stage issues the loads of all its items before it uses any of them, and the
-// lists that the searches walk sit in shared memory when they fit.
+// lists that the searches walk sit in shared memory when they fit.  A cluster of EV_CLUSTER CTAs
+// serves one cache: every CTA builds the (short) evicted lists for itself, the retained tokens are
+// dealt out among the CTAs, and CTA 0 alone changes what the others read (after the cluster barrier)
+// and keeps the books.
 __device__ __forceinline__ void evict_meta_body(const SvlmCacheDev& cd) {
+    const unsigned crank = cluster_ctarank();
     __shared__ long long wbuf64[2][META_WARPS];
     __shared__ long long s_gid[EV_SMEM];       // ordinals of the evicted tokens: text ring, then vision ring
     __shared__ long long s_pref[EV_SMEM + 2];  // exclusive prefix sums of their advances (n+1 entries per ring)
@@ -309,6 +324,7 @@ __device__ __forceinline__ void evict_meta_body(const SvlmCacheDev& cd) {
         lo1[t] = min(ring_n[t], max(lo0[t], ring_n[t] - (long long)win[t]));
         n_ev[t] = (int)(lo1[t] - lo0[t]);
     }
+    if (crank == 0 && threadIdx.x == 0) ctrl->evict_moved = 0;
     const bool in_smem = n_ev[0] + n_ev[1] <= EV_SMEM;
     // where the searches read the lists of ring t
     const long long* gid_list[2] = {in_smem ? s_gid : cd.ev_gid[0], in_smem ? s_gid + n_ev[0] : cd.ev_gid[1]};
@@ -338,12 +354,10 @@ __device__ __forceinline__ void evict_meta_body(const SvlmCacheDev& cd) {
                 if (in_smem) {
                     s_gid[(t ? n_ev[0] : 0) + i] = g[t];
                     s_pref[(t ? n_ev[0] + 1 : 0) + i] = ex;
-                } else {
+                } else {   // every CTA writes the same values
                     cd.ev_gid[t][i] = g[t];
                     cd.ev_pref[t][i] = ex;
                 }
-                cd.slot_gid[slot[t]] = -1;
-                cd.slot_delta[slot[t]] = 0;
             }
         }
     }
@@ -353,12 +367,22 @@ __device__ __forceinline__ void evict_meta_body(const SvlmCacheDev& cd) {
             else cd.ev_pref[t][n_ev[t]] = freed[t];
         }
     __syncthreads();
+    cluster_barrier();   // every CTA has read the control block and the evicted slots' metadata
+    if (crank == 0) {    // now the evicted slots can be marked empty
+        for (int t = 0; t < 2; ++t)
+            for (int i = tid; i < n_ev[t]; i += META_THREADS) {
+                const int slot = ring_slot(cd, t, lo0[t] + i);
+                cd.slot_gid[slot] = -1;
+                cd.slot_delta[slot] = 0;
+            }
+    }
 
-    // retained tokens: sinks, then the kept suffix of each ring
+    // retained tokens: sinks, then the kept suffix of each ring; CTA r takes every EV_CLUSTER-th block of them
     const long long kept_ring[2] = {ring_n[0] - lo1[0], ring_n[1] - lo1[1]};
     const long long n_kept = sink_fill + kept_ring[0] + kept_ring[1];
     int moved = 0;
-    for (long long base = 0; base < n_kept; base += (long long)KEPT_BATCH * META_THREADS) {
+    for (long long base = (long long)crank * KEPT_BATCH * META_THREADS; base < n_kept;
+         base += (long long)EV_CLUSTER * KEPT_BATCH * META_THREADS) {
         int slot[KEPT_BATCH];
         long long g[KEPT_BATCH];
         int E[KEPT_BATCH], c[KEPT_BATCH][3];
@@ -396,6 +420,9 @@ __device__ __forceinline__ void evict_meta_body(const SvlmCacheDev& cd) {
         }
     }
     if (moved) s_moved = 1;
+    __syncthreads();
+    if (tid == 0 && s_moved) atomicOr(&ctrl->evict_moved, 1);
+    if (crank != 0) return;
 
     // release the pages that fell wholly below the new low-water mark (text ring's first, in ring order)
     {
@@ -418,7 +445,6 @@ __device__ __forceinline__ void evict_meta_body(const SvlmCacheDev& cd) {
         ctrl->ring_lo[1] = lo1[1];
         ctrl->shift_total += freed[0] + freed[1];
         ctrl->n_stored = (int)n_kept;
-        ctrl->evict_moved = s_moved;
     }
 }
 
@@ -440,8 +466,25 @@ __global__ void __launch_bounds__(META_THREADS) append_meta_batch_kernel(SvlmCac
 
 __global__ void __launch_bounds__(META_THREADS) evict_meta_batch_kernel(SvlmCacheList list) {
     __shared__ SvlmCacheDev s_cd;
-    svlm_load_desc(&s_cd, list.cd[blockIdx.x]);
+    svlm_load_desc(&s_cd, list.cd[blockIdx.x / EV_CLUSTER]);
     evict_meta_body(s_cd);
+}
+
+// Launch `clusters` clusters of EV_CLUSTER CTAs.
+template <typename... Args>
+void launch_evict_meta(void (*kernel)(Args...), int clusters, cudaStream_t st, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(EV_CLUSTER * clusters);
+    cfg.blockDim = dim3(META_THREADS);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = EV_CLUSTER;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaLaunchKernelEx(&cfg, kernel, args...);
 }
 
 }  // namespace
@@ -453,7 +496,7 @@ void svlm_launch_append_meta_batch(const SvlmCacheList& list, const unsigned cha
 }
 
 void svlm_launch_evict_meta_batch(const SvlmCacheList& list, cudaStream_t st) {
-    evict_meta_batch_kernel<<<list.n, META_THREADS, 0, st>>>(list);
+    launch_evict_meta(evict_meta_batch_kernel, list.n, st, list);
     svlm_count_launch();
 }
 
@@ -464,6 +507,6 @@ void svlm_launch_append_meta(const SvlmCacheDev& cd, const unsigned char* types,
 }
 
 void svlm_launch_evict_meta(const SvlmCacheDev& cd, cudaStream_t st) {
-    evict_meta_kernel<<<1, META_THREADS, 0, st>>>(cd);
+    launch_evict_meta(evict_meta_kernel, 1, st, cd);
     svlm_count_launch();
 }
