@@ -283,12 +283,13 @@ def prefill_flops(wl, n_q, lk):
 
 
 # ------------------------------------------------------------------------------------------------
-def oracle_sample(wl, rows=48, decode=2):
-    """Times the CPU checker, as it stands, on a bounded sample of one steady-state step: one layer,
+def oracle_sample(wl, rows=1 << 20, decode=1 << 20, layers=2):
+    """Times the CPU checker, as it stands, on a bounded sample of one steady-state step: `layers` layers,
     `rows` query rows of the chunk prefill and `decode` decode steps; the rest is scaled linearly."""
     import oracle
     stream = sg.Stream(wl, 0)
-    ref = oracle.Oracle(1, wl.kv_heads, wl.head_dim, wl.n_sink, wl.vision_window, wl.text_window,
+    layers = min(layers, wl.layers)
+    ref = oracle.Oracle(layers, wl.kv_heads, wl.head_dim, wl.n_sink, wl.vision_window, wl.text_window,
                         rope_mode=wl.rope_mode, rope_base=wl.rope_base, sections=wl.sections)
     n_text, chunks = 0, 0
     while n_text < wl.n_sink + wl.text_window + 64 or chunks * wl.vision_per_chunk < wl.vision_window + 1:
@@ -303,27 +304,34 @@ def oracle_sample(wl, rows=48, decode=2):
     gids, types, pos = stream.next_chunk()
     ref.append(None, None, types, pos)
     kept = ref.query()["gids"]
-    ref.set_kv(0, kept, stream.k(0, kept), stream.v(0, kept))
-    Q = stream.q(0, gids)
+    for l in range(layers):
+        ref.set_kv(l, kept, stream.k(l, kept), stream.v(l, kept))
+    rows, decode = min(rows, len(gids)), min(decode, wl.decode_steps)
     sel = np.linspace(0, len(gids) - 1, rows).astype(np.int64)
     t0 = time.perf_counter()
     ref.evict()
     t_evict = time.perf_counter() - t0
-    t0 = time.perf_counter()
-    ref.attend(0, Q, pos, sel)
-    t_rows = time.perf_counter() - t0
+    t_rows = 0.0
+    for l in range(layers):
+        Q = stream.q(l, gids)
+        t0 = time.perf_counter()
+        ref.attend(l, Q, pos, sel)
+        t_rows += time.perf_counter() - t0
+    t_rows /= layers
     t_dec = 0.0
     for _ in range(decode):
         g1, t1, p1 = stream.next_decode_token()
-        ref.append(stream.k(0, g1)[None], stream.v(0, g1)[None], t1, p1)
-        t0 = time.perf_counter()
-        ref.attend(0, stream.q(0, g1), p1)
-        t_dec += time.perf_counter() - t0
-    t_dec /= max(decode, 1)
+        ref.append(np.stack([stream.k(l, g1) for l in range(layers)]), np.stack([stream.v(l, g1) for l in range(layers)]), t1, p1)
+        for l in range(layers):
+            q1 = stream.q(l, g1)
+            t0 = time.perf_counter()
+            ref.attend(l, q1, p1)
+            t_dec += time.perf_counter() - t0
+    t_dec /= max(decode * layers, 1)
     # one step = evict (metadata, shared by the layers) + layers x (prefill of all rows + decode steps)
     est = t_evict + wl.layers * (t_rows * len(gids) / rows + wl.decode_steps * t_dec)
-    return dict(step_seconds=est, measured_seconds=t_evict + t_rows + t_dec * decode, cores=oracle.threads(),
-                sample=f"1 of {wl.layers} layers, {rows} of {len(gids)} prefill rows, {decode} of {wl.decode_steps} "
+    return dict(step_seconds=est, measured_seconds=t_evict + (t_rows + t_dec * decode) * layers, cores=oracle.threads(),
+                sample=f"{layers} of {wl.layers} layers, {rows} of {len(gids)} prefill rows, {decode} of {wl.decode_steps} "
                        f"decode steps of one steady-state chunk; scaled linearly to the full step")
 
 
@@ -532,6 +540,109 @@ def bench_multi_stream(args, wl, base, config, peaks, rank, world, local):
                               state=dict(fill_chunks=fill_chunks, cuda_graph=True))))
 
 
+def overlap_window(wl, stream_id=0):
+    """The tokens a sliding window WITH overlap holds in one second of the stream: what the policy retains once
+    the second's chunk has been appended (the chunk included), in stream order.  Returns (gids, types, pos[n,3] or [n]) with positions counted from 0."""
+    from paper_2510_09608_b200 import binding
+    one = dataclasses_replace(wl, layers=1)
+    stream = sg.Stream(one, stream_id)
+    cache = binding.Cache(1, wl.kv_heads, wl.head_dim, wl.n_sink, wl.vision_window, wl.text_window, wl.capacity)
+    cache.set_rope(wl.rope_mode, wl.rope_base, wl.sections)
+    fill_to_steady_state(cache, one, stream)
+    import torch
+    gids, types, pos = stream.next_chunk()
+    z = torch.zeros(1, len(gids), wl.kv_heads, wl.head_dim, dtype=torch.bfloat16, device="cuda")
+    cache.append(-1, z, z, torch.from_numpy(types).cuda(), torch.from_numpy(np.ascontiguousarray(pos)).cuda())
+    cache.evict()
+    q = cache.query()
+    cache.close()
+    p = q["pos"] if wl.rope_mode else q["pos"][:, 0]
+    return q["gids"], q["types"], np.ascontiguousarray(p - p.min()).astype(np.int32)
+
+
+def bench_overlap(args, wl, base, peaks, rank, world, local):
+    """The comparison shape of the paper's efficiency argument (Figure 1(c), Section 3.3): a sliding window WITH
+    overlap recomputes the whole window every second instead of reusing the retained KV.  A step drops the cache
+    and, layer by layer, appends and chunk-prefills all R window tokens (Lq = Lk) through the same kernels."""
+    import torch
+    from paper_2510_09608_b200 import binding
+    gids, types, pos = overlap_window(wl, rank)
+    n = len(gids)
+    span = int(pos.max()) + 1
+    L = wl.layers
+    cap = (n + 127) // 128 * 128
+    cache = binding.Cache(L, wl.kv_heads, wl.head_dim, 0, 0, 0, cap)     # nothing is kept from one second to the next
+    cache.set_rope(wl.rope_mode, wl.rope_base, wl.sections)
+    gen = lambda tensor, heads: torch.stack(  # noqa: E731
+        [sg.rows_bf16_torch(wl.seed, tensor, rank, l, gids, heads, wl.head_dim) for l in range(L)])
+    K, V, Q = gen(sg.TENSOR_K, wl.kv_heads), gen(sg.TENSOR_V, wl.kv_heads), gen(sg.TENSOR_Q, wl.q_heads)
+    out = torch.empty_like(Q)
+    ty = torch.from_numpy(types).cuda()
+    total = args.warmup + args.steps + 1
+    # the window of second t sits at native positions t*span ..: the stream goes on, the contents are re-drawn
+    poss = [torch.from_numpy(np.ascontiguousarray(pos + t * span)).cuda() for t in range(total)]
+
+    def step(t, timers=None):
+        def timed(name, fn):
+            if timers is None:
+                return fn()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            fn()
+            b.record()
+            timers.setdefault(name, []).append((a, b))
+        timed("evict", cache.evict)
+        for l in range(L):
+            timed("append", lambda: cache.append(l, K[l], V[l], ty if l == 0 else None, poss[t] if l == 0 else None))
+            timed("prefill", lambda: cache.attend(l, Q[l], poss[t], out[l]))
+
+    step(0)
+    torch.cuda.synchronize()
+    assert cache.status() == binding.OK
+    graphs = []
+    cur = torch.cuda.current_stream()
+    launches = 0
+    for t in range(1, total - 1):
+        g = torch.cuda.CUDAGraph()
+        before = binding.launch_count()
+        with torch.cuda.graph(g):
+            cache.set_stream(torch.cuda.current_stream())
+            step(t)
+        launches = binding.launch_count() - before
+        graphs.append(g)
+    cache.set_stream(cur)
+    for i in range(args.warmup - 1):
+        graphs[i].replay()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local)
+    sampler.start()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    for g in graphs[args.warmup - 1:]:
+        g.replay()
+    ev1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.finish()
+    ms_per_step = max_over_ranks(ev0.elapsed_time(ev1), world) / args.steps
+    timers = {}
+    step(total - 1, timers)
+    torch.cuda.synchronize()
+    assert cache.status() == binding.OK
+    avg = {k: statistics.mean(a.elapsed_time(b) for a, b in v) for k, v in timers.items()}
+    flops = 4.0 * wl.q_heads * wl.head_dim * (n * (n + 1) / 2)
+    roof = dict(bound="tensor", kernel="prefill", achieved=flops / (avg["prefill"] * 1e-3) / 1e12, peak=peaks["bf16_burst"],
+                unit="TFLOP/s", traffic=None, algorithmic=flops, avg_ms=avg["prefill"], peak_source=peaks["source"] + " (burst bf16)")
+    roof["frac"] = roof["achieved"] / roof["peak"]
+    if rank == 0:
+        print(json.dumps(dict(base, value=whole_job_value(world, wl.frames, ms_per_step), ms_per_step=ms_per_step,
+                              config=dict(workload=f"sliding window with overlap on the config {args.config} shape: all {n} window tokens "
+                                                   f"(the retained set, newest chunk included) appended and prefilled again every second, "
+                                                   f"{L} layers, causal, Lq = Lk = {n}",
+                                          l2="Q and out of a layer (139 MB each) exceed L2; no flush", replicas="independent streams, no collective"),
+                              roofline=roof, cpu_baseline=None, e2e=None, gpu_launches=int(launches * args.steps), clocks=clocks,
+                              kernels={k: dict(avg_ms=v) for k, v in avg.items()})))
+
+
 def dataclasses_replace(obj, **kw):
     import dataclasses
     return dataclasses.replace(obj, **kw)
@@ -549,6 +660,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="replay nothing: plain calls in the timed region")
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (smaller case for profiling)")
+    ap.add_argument("--workload", default="step", choices=["step", "overlap"],
+                    help="step: the per-chunk KV-cache step (default); overlap: the whole window re-prefilled every second")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -575,7 +688,7 @@ def main():
         vals = []
         info = None
         for i in range(args.warmup + args.steps):
-            info = oracle_sample(wl, rows=16, decode=1)
+            info = oracle_sample(wl, rows=16, decode=1, layers=1)
             if i >= args.warmup:
                 vals.append(info["step_seconds"])
         sec = statistics.mean(vals)
@@ -600,6 +713,11 @@ def main():
         torch.cuda.synchronize()
 
     peaks = load_peaks()
+    if args.workload == "overlap":
+        bench_overlap(args, wl, base, peaks, rank, world, local)
+        if world > 1:
+            dist.destroy_process_group()
+        return
     if wl.streams > 1 and wl.layers == 1:
         bench_batched_decode(args, wl, base, peaks, rank, world, local)
         if world > 1:

@@ -267,3 +267,38 @@ def test_config2_whole_600_chunk_stream_metadata_and_final_outputs():
         _close(o, ref.attend(0, stream.q(0, g1), p1), "decode after 600 chunks")
     _same_metadata(cache, ref)
     _check_kv(cache, ref, stream, wl, 0, n_evicts)
+
+
+def test_overlap_workload_whole_window_reprefilled():
+    """The sliding-window-with-overlap shape of the benchmark's second workload: all 9216 tokens of one second's
+    window are appended and chunk-prefilled at once (Lq = Lk, every page causal), twice in a row with an eviction
+    that drops everything in between (more evicted tokens than the metadata kernel keeps in shared memory).
+    Sampled rows of the second pass against the checker; metadata bit-exact."""
+    import bench
+    import oracle
+    from harness import bits_to_dev, dev_to_f64
+    from paper_2510_09608_b200 import binding, streamgen as sg
+    wl = dataclasses.replace(sg.workloads()[3], layers=1)
+    gids, types, pos = bench.overlap_window(wl)
+    n = len(gids)
+    assert n == wl.retained          # the window after the second's eviction: the new chunk plus the retained history
+    span = int(pos.max()) + 1
+    cap = (n + 127) // 128 * 128
+    cache = binding.Cache(1, wl.kv_heads, wl.head_dim, 0, 0, 0, cap)
+    cache.set_rope(wl.rope_mode, wl.rope_base, wl.sections)
+    ref = oracle.Oracle(1, wl.kv_heads, wl.head_dim, 0, 0, 0, rope_mode=wl.rope_mode, rope_base=wl.rope_base, sections=wl.sections)
+    stream = sg.Stream(wl, 0)
+    K, V, Q = stream.k(0, gids), stream.v(0, gids), stream.q(0, gids)
+    ty = torch.from_numpy(types).cuda()
+    for t in range(2):
+        p = np.ascontiguousarray(pos + t * span)
+        cache.evict()
+        ref.evict()
+        cache.append(0, bits_to_dev(K), bits_to_dev(V), ty, torch.from_numpy(p).cuda())
+        ref.append(K[None], V[None], types, p)
+        out = cache.attend(0, bits_to_dev(Q), torch.from_numpy(p).cuda())
+        assert cache.status() == binding.OK
+        _same_metadata(cache, ref)
+    rng = np.random.default_rng(wl.seed)
+    rows = np.unique(np.concatenate([[0, 1, 127, 128, n - 1], rng.integers(0, n, 16)]))
+    _close(dev_to_f64(out)[rows], ref.attend(0, Q, p, rows), "whole-window prefill")
