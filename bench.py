@@ -643,6 +643,67 @@ def bench_overlap(args, wl, base, peaks, rank, world, local):
                               kernels={k: dict(avg_ms=v) for k, v in avg.items()})))
 
 
+def bench_sweep(args, wl, base, peaks, rank, world, local):
+    """Latency over the sink / text-window / vision-window values of the paper's ablations (Section 4.4: sink and
+    text window 0..1024 tokens, vision window 0..32 s), one axis at a time around the deployed policy, on the
+    config's head shape with `--layers` layers (default 4).  Per point: steady state, three steps of plain calls
+    with CUDA events around every call.  One JSON line; `value` is the deployed policy's frames/s by these timings."""
+    import torch
+    from paper_2510_09608_b200 import binding
+    L = args.layers or 4
+    per_s = wl.vision_per_chunk          # vision tokens per second of video
+    points = [("deployed", wl.n_sink, wl.text_window, wl.vision_window)]
+    points += [("sink", v, wl.text_window, wl.vision_window) for v in (0, 64, 256, 1024)]
+    points += [("text_window", wl.n_sink, v, wl.vision_window) for v in (0, 64, 256, 1024)]
+    points += [("vision_window", wl.n_sink, wl.text_window, sec * per_s) for sec in (0, 1, 4, 8, 32)]
+    rows = []
+    for axis, S, Tw, Vw in points:
+        w = dataclasses_replace(wl, layers=L, n_sink=S, text_window=Tw, vision_window=Vw)
+        stream = sg.Stream(w, rank)
+        cache = binding.Cache(L, w.kv_heads, w.head_dim, S, Vw, Tw, w.capacity)
+        cache.set_rope(w.rope_mode, w.rope_base, w.sections)
+        fill_to_steady_state(cache, w, stream)
+        cache.evict()
+        timers = {}
+        n_q = []
+        for i in range(4):
+            inp = StepInputs(w, stream, *next_step_schedule(stream, w))
+            if i == 0:
+                run_step(cache, w, inp)          # warm-up step
+                continue
+            run_step(cache, w, inp, timers)
+            n_q.append(inp.n)
+        torch.cuda.synchronize()
+        assert cache.status() == binding.OK
+        kept = len(cache.query()["gids"])
+        cache.close()
+        avg = {k: statistics.mean(a.elapsed_time(b) for a, b in v) for k, v in timers.items()}
+        tot = {k: sum(a.elapsed_time(b) for a, b in v) / 3 for k, v in timers.items()}
+        lk = kept - w.decode_steps                       # keys at the time of the chunk prefill
+        nq = int(round(statistics.mean(n_q)))
+        flops = prefill_flops(w, nq, lk) if lk >= nq else float("nan")   # the chunk itself is (partly) evicted: no closed form
+        kv_bytes = kept * 2 * w.kv_heads * w.head_dim * 2
+        moved = max(kept - w.decode_steps - S, 0)
+        ev_bytes = 2 * moved * w.kv_heads * w.head_dim * 2 * L
+        step_ms = sum(tot.values())
+        rows.append(dict(axis=axis, n_sink=S, text_window=Tw, vision_window_s=Vw // per_s, kept_tokens=kept,
+                         step_ms=step_ms, evict_ms=avg["evict"], prefill_ms=avg["prefill"],
+                         decode_layer_step_ms=avg["decode_token"] / L,
+                         prefill_frac=(flops / (avg["prefill"] * 1e-3) / 1e12 / peaks["bf16_burst"]) if flops == flops else None,
+                         decode_frac=kv_bytes * L / (avg["decode_token"] * 1e-3) / 1e9 / peaks["hbm"],
+                         evict_frac=ev_bytes / (avg["evict"] * 1e-3) / 1e9 / peaks["hbm"]))
+    if rank == 0:
+        d = rows[0]
+        roof = dict(bound="hbm", kernel="decode", achieved=d["decode_frac"] * peaks["hbm"], peak=peaks["hbm"], unit="GB/s",
+                    frac=d["decode_frac"], traffic=None, peak_source=peaks["source"] + " (copy)")
+        print(json.dumps(dict(base, value=wl.frames / (d["step_ms"] * 1e-3), ms_per_step=d["step_ms"],
+                              config=dict(workload=f"policy sweep on the config {args.config} shape, {L} layers: one axis at a time around "
+                                                   f"sinks {wl.n_sink} / text {wl.text_window} / vision {wl.vision_window // per_s} s; plain calls, event-timed",
+                                          l2="no flush: the layers' K/V in turn exceed L2 except at the smallest windows (see kept_tokens)",
+                                          replicas="independent streams, no collective"),
+                              roofline=roof, cpu_baseline=None, e2e=None, gpu_launches=None, clocks=None, sweep=rows)))
+
+
 def dataclasses_replace(obj, **kw):
     import dataclasses
     return dataclasses.replace(obj, **kw)
@@ -660,8 +721,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="replay nothing: plain calls in the timed region")
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (smaller case for profiling)")
-    ap.add_argument("--workload", default="step", choices=["step", "overlap"],
-                    help="step: the per-chunk KV-cache step (default); overlap: the whole window re-prefilled every second")
+    ap.add_argument("--workload", default="step", choices=["step", "overlap", "sweep"],
+                    help="step: the per-chunk KV-cache step (default); overlap: the whole window re-prefilled every second; "
+                         "sweep: the step's latency over the paper's sink / window ablation values")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -713,6 +775,11 @@ def main():
         torch.cuda.synchronize()
 
     peaks = load_peaks()
+    if args.workload == "sweep":
+        bench_sweep(args, sg.workloads()[args.config], base, peaks, rank, world, local)
+        if world > 1:
+            dist.destroy_process_group()
+        return
     if args.workload == "overlap":
         bench_overlap(args, wl, base, peaks, rank, world, local)
         if world > 1:
