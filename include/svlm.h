@@ -151,6 +151,17 @@ int svlm_attend_batched(svlm_cache* const* caches, int n_caches, int layer, cons
                         int n_q, int q_heads, void* out);
 
 /*
+ * svlm_attend_batched for streams whose new chunks differ in length (each second's text burst varies):
+ * cache i attends with its last n_q[i] appended tokens, n_q a HOST array of n_caches counts >= 1.
+ * Q, out are [sum n_q][q_heads][head_dim], q_pos [sum n_q] or [sum n_q][3]: the caches' rows one after
+ * another in the order of `caches`.  One chunk-prefill launch serves all caches (also rows-of-one
+ * caches: the split-KV decode path is not taken here).  layer >= 0 only.
+ * Errors: as svlm_attend_batched; SVLM_ERR_ARG for a repeated cache or a count below 1.
+ */
+int svlm_attend_batched_varlen(svlm_cache* const* caches, int n_caches, int layer, const void* Q, const int32_t* q_pos,
+                               const int32_t* n_q, int q_heads, void* out);
+
+/*
  * Batched forms for independent streams that advance in lock step (one generated token per stream per
  * step, as in batched serving; the paper's policy is per stream, so each cache behaves exactly as under
  * the single-cache calls).  Same requirements on the caches as svlm_attend_batched; a cache may appear

@@ -36,6 +36,7 @@ _lib.svlm_cache_evict.argtypes = [_vp]
 _lib.svlm_attend.argtypes = [_vp, _i, _vp, _vp, _i, _i, _vp]
 _lib.svlm_decode_step.argtypes = [_vp, _i, _vp, _vp, _vp, _vp, _vp, _i, _vp]
 _lib.svlm_attend_batched.argtypes = [C.POINTER(_vp), _i, _i, _vp, _vp, _i, _i, _vp]
+_lib.svlm_attend_batched_varlen.argtypes = [C.POINTER(_vp), _i, _i, _vp, _vp, C.POINTER(C.c_int32), _i, _vp]
 _lib.svlm_decode_step_batched.argtypes = [C.POINTER(_vp), _i, _i, _vp, _vp, _vp, _vp, _vp, _i, _vp]
 _lib.svlm_cache_evict_batched.argtypes = [C.POINTER(_vp), _i]
 _lib.svlm_cache_append_host.argtypes = [_vp, _i, _vp, _vp, _vp, _vp, _i]
@@ -202,6 +203,19 @@ def attend_batched(caches, layer, Q, q_pos, out=None):
     rc = _lib.svlm_attend_batched(arr, len(caches), layer, _dev_ptr(Q, torch.bfloat16), _dev_ptr(q_pos, torch.int32),
                                   Q.shape[1], Q.shape[2], _dev_ptr(out, torch.bfloat16))
     _check(rc, "svlm_attend_batched")
+    return out
+
+
+def attend_batched_varlen(caches, layer, Q, q_pos, n_q, out=None):
+    """Chunk prefill of several caches whose chunks differ in length, one launch: Q [sum(n_q), q_heads, d] bf16 CUDA with
+    the caches' rows one after another, q_pos likewise, n_q a sequence of ints (svlm_attend_batched_varlen)."""
+    if out is None:
+        out = torch.empty_like(Q)
+    arr = (_vp * len(caches))(*[c._h for c in caches])
+    cnt = (C.c_int32 * len(caches))(*[int(x) for x in n_q])
+    rc = _lib.svlm_attend_batched_varlen(arr, len(caches), layer, _dev_ptr(Q, torch.bfloat16), _dev_ptr(q_pos, torch.int32), cnt,
+                                         Q.shape[1], _dev_ptr(out, torch.bfloat16))
+    _check(rc, "svlm_attend_batched_varlen")
     return out
 
 

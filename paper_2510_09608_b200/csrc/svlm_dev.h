@@ -104,6 +104,9 @@ struct SvlmAttendBatch {     // kernel parameter: up to 32 caches share one laun
     int layers, kv_heads, head_dim, n_slots;
     int rope_mode, sec_t, sec_th;
     SvlmAttendView view[SVLM_MAX_BATCH];
+    int q_varlen;            // chunk prefill only: the caches bring different numbers of query rows,
+    int q_off[SVLM_MAX_BATCH];   //   cache i's rows start at row q_off[i] of Q, q_pos and out
+    int q_cnt[SVLM_MAX_BATCH];   //   and there are q_cnt[i] of them
     const float* rope_tab;   // rotation table of the first cache (all caches of a batch share the geometry)
     double theta[SVLM_MAX_HALF];
 };

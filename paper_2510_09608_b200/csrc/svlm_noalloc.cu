@@ -88,6 +88,7 @@ extern "C" int svlm_attend_decode_noalloc(svlm_cache* c, int layer, const void* 
         SvlmAttendView& v = b.view[0];
         v.K = d.K; v.V = d.V; v.ctrl = d.ctrl; v.tiles = d.tiles; v.slot_gid = d.slot_gid; v.tmaps = d.tmaps; v.new_slot = d.new_slot; v.slot_c = d.slot_c;
         b.rope_tab = d.rope_tab;
+        b.q_varlen = 0;
         v.ws = scratch;
         if (svlm_launch_decode(b, layer, 1, Q, q_pos, q_heads, out, splits, nullptr, nullptr, 0, c->stream) != cudaSuccess)
             rc = SVLM_ERR_CUDA;

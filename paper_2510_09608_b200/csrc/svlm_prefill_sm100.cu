@@ -236,7 +236,7 @@ static_assert(sizeof(PfShared) <= 2040, "control block must leave room for the t
 template <int D>
 __global__ void __launch_bounds__(PF_THREADS, 1)
 prefill_kernel(SvlmAttendBatch b, int layer0, int n_layers, const uint16_t* __restrict__ Q,
-               const int* __restrict__ q_pos, int n_q, int q_heads, uint16_t* __restrict__ out) {
+               const int* __restrict__ q_pos, int n_q_arg, int q_heads, uint16_t* __restrict__ out) {
     constexpr int KB = D / 64;                 // 64-element (128-byte) blocks along d
     constexpr int TILE_BYTES = 128 * D * 2;    // one K or V page of one head, or one 128-row Q tile
     constexpr int HALF = D / 2;
@@ -254,6 +254,11 @@ prefill_kernel(SvlmAttendBatch b, int layer0, int n_layers, const uint16_t* __re
     const int ci = prob / n_layers, li = prob % n_layers;
     const int layer = layer0 + li;
     const SvlmAttendView& vw = b.view[ci];
+    // rows of this problem: n_q_arg per problem, or (caches with chunks of different lengths) the cache's own count
+    const int n_q = b.q_varlen ? b.q_cnt[ci] : n_q_arg;
+    const size_t q_row0 = b.q_varlen ? (size_t)b.q_off[ci] : (size_t)prob * n_q_arg;   // first row in Q and out
+    const size_t p_row0 = b.q_varlen ? (size_t)b.q_off[ci] : (size_t)ci * n_q_arg;     // first row in q_pos
+    if ((int)(blockIdx.x >> 1) * PF_ROWS >= n_q * G) return;   // a shorter chunk: both CTAs of the pair leave at once
     const int m_total = n_q * G;
     const unsigned rank = cluster_rank();      // which half of the pages this CTA takes
     const int m0 = (blockIdx.x >> 1) * PF_ROWS;
@@ -339,7 +344,7 @@ prefill_kernel(SvlmAttendBatch b, int layer0, int n_layers, const uint16_t* __re
                 if (i < n_ent) {
                     const int tk = i / HALF, pair = i % HALF;
                     const int axis = b.rope_mode == 0 ? 0 : (pair < b.sec_t ? 0 : (pair < b.sec_th ? 1 : 2));
-                    cpos[u] = (long long)__ldg(q_pos + ((size_t)ci * n_q + r_lo + tk) * pw + axis) - shift;
+                    cpos[u] = (long long)__ldg(q_pos + (p_row0 + r_lo + tk) * pw + axis) - shift;
                 }
             }
 #pragma unroll
@@ -375,7 +380,7 @@ prefill_kernel(SvlmAttendBatch b, int layer0, int n_layers, const uint16_t* __re
                 const bool live = mg < m_total;
                 const int r = live ? mg / G : r_lo, h = live ? mg % G : 0;
                 tok[u] = r;
-                const uint4* src = reinterpret_cast<const uint4*>(Q + ((((size_t)prob) * n_q + r) * q_heads + hk * G + h) * D);
+                const uint4* src = reinterpret_cast<const uint4*>(Q + ((q_row0 + r) * q_heads + hk * G + h) * D);
                 lo4[u] = live ? __ldg(src + c8v[u]) : make_uint4(0, 0, 0, 0);
                 hi4[u] = live ? __ldg(src + CH + c8v[u]) : make_uint4(0, 0, 0, 0);
             }
@@ -383,7 +388,7 @@ prefill_kernel(SvlmAttendBatch b, int layer0, int n_layers, const uint16_t* __re
             for (int u = 0; u < UN; ++u) {
                 const int c8 = c8v[u], g = row[u] >> 7, m = row[u] & 127;
                 const float2* cs_row = s_cs + (size_t)(tok[u] - r_lo) * HALF;
-                const int* qp = q_pos + ((size_t)ci * n_q + tok[u]) * (b.rope_mode == 0 ? 1 : 3);
+                const int* qp = q_pos + (p_row0 + tok[u]) * (b.rope_mode == 0 ? 1 : 3);
                 const unsigned* lw = reinterpret_cast<const unsigned*>(&lo4[u]);
                 const unsigned* hw = reinterpret_cast<const unsigned*>(&hi4[u]);
                 float2 cs8[8];
@@ -610,7 +615,7 @@ prefill_kernel(SvlmAttendBatch b, int layer0, int n_layers, const uint16_t* __re
             const float inv = L > 0.f ? 1.f / L : 0.f;
             const float ga = fa * inv, gb = fb * inv;
             const bool live = mg < m_total;
-            uint16_t* dst = out + ((((size_t)prob) * n_q + r) * q_heads + hk * G + (mg % G)) * D;
+            uint16_t* dst = out + ((q_row0 + r) * q_heads + hk * G + (mg % G)) * D;
 #pragma unroll 1
             for (int q4 = 0; q4 < D / 32; ++q4) {
                 float o[32];

@@ -133,6 +133,7 @@ void fill_batch_geometry(const svlm_cache* c, SvlmAttendBatch& b) {
     b.sec_th = c->dev.sec_th;
     std::memcpy(b.theta, c->dev.theta, sizeof b.theta);
     b.rope_tab = c->dev.rope_tab;
+    b.q_varlen = 0;
 }
 
 // Caches that may share one launch: same shape, rotary settings and device.
@@ -445,6 +446,36 @@ int svlm_decode_step_batched(svlm_cache* const* caches, int n_caches, int layer,
             if (caches[i]->pending_n != 1) return SVLM_ERR_ORDER;
     }
     return attend_common(caches, n_caches, layer, Q, pos, 1, q_heads, out, K, V);
+}
+
+int svlm_attend_batched_varlen(svlm_cache* const* caches, int n_caches, int layer, const void* Q, const int32_t* q_pos,
+                               const int32_t* n_q, int q_heads, void* out) {
+    SvlmCacheList list;   // only for its checks: distinct caches of one geometry
+    int rc = make_list(caches, n_caches, list);
+    if (rc != SVLM_OK) return rc;
+    svlm_cache* c0 = caches[0];
+    if (!Q || !q_pos || !n_q || !out || q_heads < 1 || layer < 0 || layer >= c0->dev.layers) return SVLM_ERR_ARG;
+    if (q_heads % c0->dev.kv_heads || !svlm_prefill_supported(c0->dev.n_pages, q_heads / c0->dev.kv_heads)) return SVLM_ERR_ARG;
+    SvlmAttendBatch b;
+    b.n_caches = n_caches;
+    fill_batch_geometry(c0, b);
+    b.q_varlen = 1;
+    long long off = 0;
+    int n_max = 0;
+    for (int i = 0; i < n_caches; ++i) {
+        if (n_q[i] < 1) return SVLM_ERR_ARG;
+        if (n_q[i] > caches[i]->appended) return SVLM_ERR_ORDER;
+        b.q_off[i] = (int)off;
+        b.q_cnt[i] = n_q[i];
+        off += n_q[i];
+        n_max = std::max(n_max, n_q[i]);
+        fill_view(caches[i], b.view[i]);
+        caches[i]->last_decode_layer = -1;
+    }
+    if (off > 0x7fffffffll) return SVLM_ERR_ARG;
+    DeviceGuard guard(c0->device);
+    SVLM_CUDA(svlm_launch_prefill(b, layer, 1, Q, q_pos, n_max, q_heads, out, c0->stream));
+    return SVLM_OK;
 }
 
 int svlm_attend_batched(svlm_cache* const* caches, int n_caches, int layer, const void* Q, const int32_t* q_pos,

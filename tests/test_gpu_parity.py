@@ -197,6 +197,37 @@ def test_batched_decode_steps_and_batched_evict(rope_1d):
     assert e.value.status == binding.ERR_ARG
 
 
+def test_batched_chunk_prefill_with_chunks_of_different_lengths():
+    """svlm_attend_batched_varlen: four streams whose new chunks differ in length (one contributes a single row)
+    attend in one launch per layer; every output row of every stream against the checker."""
+    from harness import SideBySide, assert_close, bits_to_dev, dev_to_f64
+    from paper_2510_09608_b200 import binding
+    wl = dataclasses.replace(_wl(2), layers=2, n_sink=16, vision_window=320, text_window=40, frames=1, grid_h=8, grid_w=8)
+    sides = [SideBySide(wl, stream=i) for i in range(4)]
+    for i, s in enumerate(sides):
+        for _ in range(2 + 2 * i):
+            s.append_chunk()
+            s.evict()
+        s.append_chunk()
+        s.evict()
+    sides[3].append_decode_token()                       # this stream attends with one row only
+    n_q = [len(s.last[0]) for s in sides]
+    assert len(set(n_q)) > 2 and n_q[3] == 1
+    pos = torch.from_numpy(np.ascontiguousarray(np.concatenate([s.last[2] for s in sides]))).cuda()
+    for l in range(wl.layers):
+        Q = np.concatenate([s.stream.q(l, s.last[0]) for s in sides])
+        out = dev_to_f64(binding.attend_batched_varlen([s.cache for s in sides], l, bits_to_dev(Q), pos, n_q))
+        o = 0
+        for s, n in zip(sides, n_q):
+            assert s.cache.status() == binding.OK
+            s._give_values_to_ref(l)
+            assert_close(s._stats(out[o:o + n], s.ref.attend(l, Q[o:o + n], s.last[2])))
+            o += n
+    with pytest.raises(binding.SvlmError) as e:
+        binding.attend_batched_varlen([s.cache for s in sides], 0, bits_to_dev(Q), pos, [n_q[0], n_q[1], n_q[2], 0])
+    assert e.value.status == binding.ERR_ARG
+
+
 def test_errors_and_capacity():
     from paper_2510_09608_b200 import binding
     with pytest.raises(binding.SvlmError):
