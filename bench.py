@@ -180,10 +180,19 @@ def stack_decode_inputs(inps):
     return toks
 
 
-def run_step_multi(caches, wl, inps, dec, timers=None):
+def stack_prefill_inputs(inps):
+    """The streams' chunk queries one after another, per layer: Q [layers][sum n][q_heads][d], pos [sum n](x3), the
+    row counts, and an output buffer of Q's shape (the layout of svlm_attend_batched_varlen)."""
+    import torch
+    Q = torch.cat([inp.Q for inp in inps], dim=1).contiguous()
+    return dict(Q=Q, pos=torch.cat([inp.pos for inp in inps]).contiguous(), n_q=[inp.n for inp in inps], out=torch.empty_like(Q))
+
+
+def run_step_multi(caches, wl, inps, dec, timers=None, pre=None):
     """One step of several streams that advance in lock step: every stream appends its chunk, ONE batched
-    eviction, chunk prefill per stream and layer (the chunks differ in length), then the generated tokens with one
-    batched decode launch per layer for all streams.  inps: one StepInputs per stream; dec: stack_decode_inputs."""
+    eviction, per layer the streams' K/V appends and ONE chunk-prefill launch for all of them (the chunks differ in
+    length), then the generated tokens with one batched decode launch per layer for all streams.
+    inps: one StepInputs per stream; dec: stack_decode_inputs; pre: stack_prefill_inputs (outputs land in pre["out"])."""
     import torch
     from paper_2510_09608_b200 import binding
     L = wl.layers
@@ -200,11 +209,13 @@ def run_step_multi(caches, wl, inps, dec, timers=None):
     for c, inp in zip(caches, inps):
         timed("append", lambda: c.append(0, inp.K[0], inp.V[0], inp.types, inp.pos))
     timed("evict", lambda: binding.evict_batched(caches))
+    if pre is None:
+        pre = stack_prefill_inputs(inps)
     for l in range(L):
-        for c, inp in zip(caches, inps):
-            if l:
+        if l:
+            for c, inp in zip(caches, inps):
                 timed("append", lambda: c.append(l, inp.K[l], inp.V[l]))
-            timed("prefill", lambda: c.attend(l, inp.Q[l], inp.pos, inp.out[l]))
+        timed("prefill", lambda: binding.attend_batched_varlen(caches, l, pre["Q"][l], pre["pos"], pre["n_q"], pre["out"][l]))
 
     def decode_token(d):
         for l in range(L):
@@ -428,7 +439,7 @@ def bench_batched_decode(args, wl, base, peaks, rank, world, local):
 
 def bench_multi_stream(args, wl, base, config, peaks, rank, world, local):
     """Workload 5: `wl.streams` streams of a full attention stack in lock step; a step is one chunk of every stream
-    (append, batched eviction, per-stream chunk prefill, batched decode).  Steps are replayed from CUDA graphs;
+    (append, batched eviction, batched chunk prefill, batched decode).  Steps are replayed from CUDA graphs;
     value = frames/s over all streams."""
     import torch
     from paper_2510_09608_b200 import binding
@@ -446,7 +457,10 @@ def bench_multi_stream(args, wl, base, config, peaks, rank, world, local):
 
     def make_step():
         inps = [StepInputs(wl, st, *next_step_schedule(st, wl)) for st in streams]
-        return inps, stack_decode_inputs(inps)
+        pre = stack_prefill_inputs(inps)
+        for inp in inps:          # the per-stream copies of Q and the output are not needed any more
+            inp.Q = inp.out = None
+        return inps, stack_decode_inputs(inps), pre
 
     total = args.warmup + args.steps
     steps = [make_step() for _ in range(total)]
@@ -457,20 +471,20 @@ def bench_multi_stream(args, wl, base, config, peaks, rank, world, local):
         c = binding.Cache(wl.layers, wl.kv_heads, wl.head_dim, wl.n_sink, wl.vision_window, wl.text_window, wl.capacity)
         c.set_rope(wl.rope_mode, wl.rope_base, wl.sections)
         scratch.append(c)
-    run_step_multi(scratch, wl, *steps[0])
+    run_step_multi(scratch, wl, steps[0][0], steps[0][1], None, steps[0][2])
     torch.cuda.synchronize()
     for c in scratch:
         c.close()
 
     graphs, launches = [], []
     cur = torch.cuda.current_stream()
-    for inps, dec in steps:
+    for inps, dec, pre in steps:
         g = torch.cuda.CUDAGraph()
         before = binding.launch_count()
         with torch.cuda.graph(g):
             for c in caches:
                 c.set_stream(torch.cuda.current_stream())
-            run_step_multi(caches, wl, inps, dec)
+            run_step_multi(caches, wl, inps, dec, None, pre)
         launches.append(binding.launch_count() - before)
         graphs.append(g)
     for c in caches:
@@ -501,14 +515,14 @@ def bench_multi_stream(args, wl, base, config, peaks, rank, world, local):
 
     # per-kernel durations: one plain pass with events around every call
     timers = {}
-    run_step_multi(caches, wl, *prime, timers)
+    run_step_multi(caches, wl, prime[0], prime[1], timers, prime[2])
     torch.cuda.synchronize()
     kern = {k: [a.elapsed_time(b) for a, b in v] for k, v in timers.items()}
     avg = {k: statistics.mean(v) for k, v in kern.items()}
     tot = {k: sum(v) for k, v in kern.items()}
     n_q = statistics.mean(inp.n for inp in prime[0])
     lk = wl.retained
-    flops = prefill_flops(wl, int(round(n_q)), lk)
+    flops = sum(prefill_flops(wl, inp.n, lk) for inp in prime[0])          # one prefill launch: all streams, one layer
     kv_bytes_layer = lk * 2 * wl.kv_heads * wl.head_dim * 2 * S          # one batched decode launch: all streams, one layer
     evict_bytes = 2 * (wl.retained - wl.n_sink) * wl.kv_heads * wl.head_dim * 2 * wl.layers * S
     kernels = {
@@ -531,7 +545,7 @@ def bench_multi_stream(args, wl, base, config, peaks, rank, world, local):
                     peak_source=peaks["source"] + (" (burst bf16)" if dominant == "prefill" else " (copy)"))
     if rank == 0:
         config = dict(config, replicas="independent streams, no collective",
-                      streams=f"{S} streams per GPU in lock step: batched eviction and decode, per-stream prefill")
+                      streams=f"{S} streams per GPU in lock step: batched eviction, chunk prefill and decode (one launch per layer for all streams)")
         print(json.dumps(dict(base, value=whole_job_value(world, wl.frames * S, ms_per_step), ms_per_step=ms_per_step,
                               config=config, roofline=roofline, cpu_baseline=None, e2e=None,
                               gpu_launches=int(sum(launches[args.warmup:])), clocks=clocks, kernels=kernels,

@@ -184,7 +184,8 @@ def test_config4_batched_decode_16_streams_with_interleaved_eviction():
 def test_config5_high_frame_rate_streams_sampled():
     """The 8 frames/s x 8x8-grid shape (vision blocks of span 8, text bursts up to 32): three of the eight streams,
     four of the 28 layers, one steady-state step run as benchmarked: the streams advance in lock step (per-stream
-    appends and chunk prefill, one batched eviction, one batched decode launch per layer and token)."""
+    appends, one batched eviction, one chunk-prefill launch per layer for all streams' different-length chunks, one
+    batched decode launch per layer and token)."""
     import bench
     from harness import dev_to_f64
     from paper_2510_09608_b200 import streamgen as sg
@@ -199,7 +200,9 @@ def test_config5_high_frame_rate_streams_sampled():
     scheds = [bench.next_step_schedule(s, wl) for s, _, _ in sides]
     inps = [bench.StepInputs(wl, s, chunk, decode) for (s, _, _), (chunk, decode) in zip(sides, scheds)]
     dec = bench.stack_decode_inputs(inps)
-    bench.run_step_multi([c for _, c, _ in sides], wl, inps, dec)
+    pre = bench.stack_prefill_inputs(inps)
+    bench.run_step_multi([c for _, c, _ in sides], wl, inps, dec, None, pre)
+    offs = np.concatenate([[0], np.cumsum(pre["n_q"])])
     torch.cuda.synchronize()
     for i, ((stream, cache, ref), (chunk, decode), inp) in enumerate(zip(sides, scheds, inps)):
         gids, types, pos = chunk
@@ -208,7 +211,7 @@ def test_config5_high_frame_rate_streams_sampled():
         rows = np.unique(np.concatenate([[0, len(gids) - 1], rng.integers(0, len(gids), 16)]))
         for l in (0, 3):
             _give(ref, stream, l)
-            _close(dev_to_f64(inp.out[l])[rows], ref.attend(l, stream.q(l, gids), pos, rows), f"stream {i} prefill layer {l}")
+            _close(dev_to_f64(pre["out"][l][offs[i]:offs[i + 1]])[rows], ref.attend(l, stream.q(l, gids), pos, rows), f"stream {i} prefill layer {l}")
         for g1, t1, p1 in decode:
             ref.append(None, None, t1, p1)
             for l in (0, 3):
