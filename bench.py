@@ -764,7 +764,7 @@ def main():
         vals = []
         info = None
         for i in range(args.warmup + args.steps):
-            info = oracle_sample(wl, rows=16, decode=1, layers=1)
+            info = oracle_sample(wl, decode=2, layers=1)   # one whole layer of prefill rows: the per-call set-up is not scaled up
             if i >= args.warmup:
                 vals.append(info["step_seconds"])
         sec = statistics.mean(vals)
