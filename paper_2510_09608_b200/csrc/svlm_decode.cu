@@ -545,22 +545,14 @@ cudaError_t svlm_launch_decode(const SvlmAttendBatch& b, int layer0, int n_layer
     const uint16_t* Vn = (const uint16_t*)Vnew;
     cudaError_t e;
     if (b.head_dim == 128) {
-        static bool once = false;
-        if (!once) {
-            e = cudaFuncSetAttribute(decode_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)decode_smem<128>());
-            if (e != cudaSuccess) return e;
-            once = true;
-        }
+        e = svlm_allow_smem<decode_kernel<128>>(decode_smem<128>());
+        if (e != cudaSuccess) return e;
         cfg.dynamicSmemBytes = decode_smem<128>();
         e = cudaLaunchKernelEx(&cfg, decode_kernel<128>, b, layer0, n_layers, Qp, q_pos, q_heads, Op, splits, Kn, Vn,
                                early_loads);
     } else {
-        static bool once = false;
-        if (!once) {
-            e = cudaFuncSetAttribute(decode_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)decode_smem<64>());
-            if (e != cudaSuccess) return e;
-            once = true;
-        }
+        e = svlm_allow_smem<decode_kernel<64>>(decode_smem<64>());
+        if (e != cudaSuccess) return e;
         cfg.dynamicSmemBytes = decode_smem<64>();
         e = cudaLaunchKernelEx(&cfg, decode_kernel<64>, b, layer0, n_layers, Qp, q_pos, q_heads, Op, splits, Kn, Vn,
                                early_loads);

@@ -1,9 +1,26 @@
 // Host-side launchers of the kernels (one translation unit per kernel family).
 #pragma once
 #include <cuda_runtime.h>
+
+#include <atomic>
+
 #include "svlm_dev.h"
 
 void svlm_count_launch();
+
+// Raises a kernel's dynamic shared-memory limit, once per device (the attribute belongs to the device's
+// context) and safe to call from several host threads.  The current device is the one the launch goes to.
+template <auto Kernel>
+cudaError_t svlm_allow_smem(size_t bytes) {
+    static std::atomic<unsigned long long> done{0};   // one bit per device, one word per kernel instantiation
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 64 && ((done.load(std::memory_order_acquire) >> dev) & 1ull)) return cudaSuccess;
+    e = cudaFuncSetAttribute(Kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+    if (e == cudaSuccess && dev < 64) done.fetch_or(1ull << dev, std::memory_order_release);
+    return e;
+}
 
 // metadata (svlm_meta.cu)
 void svlm_launch_append_meta(const SvlmCacheDev& cd, const unsigned char* types, const int* pos, int n, cudaStream_t st);

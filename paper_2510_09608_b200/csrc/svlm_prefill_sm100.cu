@@ -673,13 +673,8 @@ constexpr size_t prefill_smem() { return sizeof(PfShared) + 1024 + (size_t)(2 + 
 template <int D>
 cudaError_t launch(const SvlmAttendBatch& b, int layer0, int n_layers, const uint16_t* Q, const int* q_pos, int n_q,
                    int q_heads, uint16_t* out, cudaStream_t st) {
-    static bool once = false;
-    cudaError_t e;
-    if (!once) {
-        e = cudaFuncSetAttribute(prefill_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)prefill_smem<D>());
-        if (e != cudaSuccess) return e;
-        once = true;
-    }
+    cudaError_t e = svlm_allow_smem<prefill_kernel<D>>(prefill_smem<D>());
+    if (e != cudaSuccess) return e;
     const int G = q_heads / b.kv_heads;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(2 * ((n_q * G + PF_ROWS - 1) / PF_ROWS), b.kv_heads, b.n_caches * n_layers);

@@ -136,9 +136,9 @@ void fill_batch_geometry(const svlm_cache* c, SvlmAttendBatch& b) {
     b.q_varlen = 0;
 }
 
-// Caches that may share one launch: same shape, rotary settings and device.
+// Caches that may share one launch: same shape, rotary settings, device and stream.
 bool same_geometry(const svlm_cache* c, const svlm_cache* c0) {
-    return c->dev.layers == c0->dev.layers && c->dev.kv_heads == c0->dev.kv_heads &&
+    return c->stream == c0->stream && c->dev.layers == c0->dev.layers && c->dev.kv_heads == c0->dev.kv_heads &&
            c->dev.head_dim == c0->dev.head_dim && c->dev.n_slots == c0->dev.n_slots &&
            c->dev.rope_mode == c0->dev.rope_mode && c->dev.sec_t == c0->dev.sec_t && c->dev.sec_th == c0->dev.sec_th &&
            c->dev.theta[1] == c0->dev.theta[1] && c->device == c0->device;

@@ -195,6 +195,12 @@ def test_batched_decode_steps_and_batched_evict(rope_1d):
     with pytest.raises(binding.SvlmError) as e:          # a cache may appear only once in a batch
         binding.evict_batched([caches[0], caches[0]])
     assert e.value.status == binding.ERR_ARG
+    side = torch.cuda.Stream()
+    caches[1].set_stream(side)                           # caches of a batch must sit on one stream
+    with pytest.raises(binding.SvlmError) as e:
+        binding.evict_batched(caches)
+    assert e.value.status == binding.ERR_ARG
+    caches[1].set_stream(torch.cuda.current_stream())
 
 
 def test_batched_chunk_prefill_with_chunks_of_different_lengths():
