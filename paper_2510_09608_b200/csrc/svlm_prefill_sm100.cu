@@ -583,19 +583,26 @@ prefill_kernel(SvlmAttendBatch b, int layer0, int n_layers, const uint16_t* __re
         tc_fence_after();
 
         // ---- hand-over between the two CTAs of the cluster, then the output ------------------------
-        // CTA k of the pair finishes tile k: its group 1-k sends (O, m, l) of its rows to the partner, its group k
-        // merges its own accumulator with what the partner's group k sent.  The exchange area is the K/V ring,
-        // idle once a CTA's MMAs have completed (cluster barrier #1 says so for both).
+        // CTA k of the pair finishes tile k.  Both warpgroups work on both steps, each on one half of the head
+        // dimension (a warp reaches its TMEM lane quadrant in either tile): first tile 1-k's (O, m, l) goes to
+        // the partner, then tile k's accumulator is merged with what the partner sent and written out.  The
+        // exchange area is the K/V ring, idle once a CTA's MMAs have completed (cluster barrier #1 says so for
+        // both); a row's (m, l) reaches the other warpgroup through the same area.
         float* xo = reinterpret_cast<float*>(ring);                      // [D/4 chunks][128 rows] float4
-        float* xml = xo + (size_t)128 * D;                               // [128 rows][2]
+        float* xml = xo + (size_t)128 * D;                               // [128 rows][2]: the partner's (m, l)
+        float2* lml = reinterpret_cast<float2*>(xml + 2 * 128);          // [2 tiles][128 rows]: this CTA's (m, l)
         const bool mine = n_proc > 0;                                    // this CTA processed pages
-        cluster_sync_all();   // #1: neither CTA needs its ring any more
-        if ((unsigned)g != rank) {
+        lml[g * 128 + m] = make_float2(ok && mine ? m_ref : -INFINITY, ok && mine ? l : 0.f);
+        cluster_sync_all();   // #1: neither CTA needs its ring any more; (m, l) of every row is visible
+        const int gk = (int)rank, gs = gk ^ 1;                           // tile kept, tile sent
+        constexpr int QH = D / 64;                                       // 32-column chunks of O per half
+        {
+            const unsigned tOs = tmem + 256 + gs * 128 + lane_base;
             const unsigned dst_o = map_to_rank(xo, rank ^ 1), dst_ml = map_to_rank(xml, rank ^ 1);
 #pragma unroll 1
-            for (int q4 = 0; q4 < D / 32; ++q4) {
+            for (int q4 = g * QH; q4 < (g + 1) * QH; ++q4) {
                 float o[32];
-                if (mine) { tmem_ld32(tO + q4 * 32, o); tmem_wait_ld(); }
+                if (mine) { tmem_ld32(tOs + q4 * 32, o); tmem_wait_ld(); }
 #pragma unroll
                 for (int i = 0; i < 8; ++i) {
                     const float4 v = mine ? make_float4(o[4 * i], o[4 * i + 1], o[4 * i + 2], o[4 * i + 3])
@@ -603,23 +610,27 @@ prefill_kernel(SvlmAttendBatch b, int layer0, int n_layers, const uint16_t* __re
                     st_cluster_v4(dst_o + (unsigned)(((q4 * 8 + i) * 128 + m) * 16), v);
                 }
             }
-            st_cluster_v2(dst_ml + (unsigned)(m * 8), make_float2(ok && mine ? m_ref : -INFINITY, ok && mine ? l : 0.f));
+            if (g == 0) st_cluster_v2(dst_ml + (unsigned)(m * 8), lml[gs * 128 + m]);
         }
         cluster_sync_all();   // #2: the partner's rows have arrived
-        if ((unsigned)g == rank && ok) {
+        if (ok) {
+            const unsigned tOk = tmem + 256 + gk * 128 + lane_base;
+            const int mgk = m0 + gk * 128 + m;
+            const int rk = min(mgk / G, n_q - 1);
             const float mb = xml[m * 2], lb = xml[m * 2 + 1];
-            const float ma = mine ? m_ref : -INFINITY, la = mine ? l : 0.f;
+            const float2 own = lml[gk * 128 + m];
+            const float ma = own.x, la = own.y;
             const float M = fmaxf(ma, mb);
             const float fa = ma == -INFINITY ? 0.f : exp2f(ma - M), fb = mb == -INFINITY ? 0.f : exp2f(mb - M);
             const float L = la * fa + lb * fb;
             const float inv = L > 0.f ? 1.f / L : 0.f;
             const float ga = fa * inv, gb = fb * inv;
-            const bool live = mg < m_total;
-            uint16_t* dst = out + ((q_row0 + r) * q_heads + hk * G + (mg % G)) * D;
+            const bool live = mgk < m_total;
+            uint16_t* dst = out + ((q_row0 + rk) * q_heads + hk * G + (mgk % G)) * D;
 #pragma unroll 1
-            for (int q4 = 0; q4 < D / 32; ++q4) {
+            for (int q4 = g * QH; q4 < (g + 1) * QH; ++q4) {
                 float o[32];
-                if (mine) { tmem_ld32(tO + q4 * 32, o); tmem_wait_ld(); }
+                if (mine) { tmem_ld32(tOk + q4 * 32, o); tmem_wait_ld(); }
 #pragma unroll
                 for (int i = 0; i < 8; ++i) {
                     const float4 pb = *reinterpret_cast<const float4*>(xo + (size_t)((q4 * 8 + i) * 128 + m) * 4);
