@@ -99,6 +99,23 @@ int svlm_cache_append(svlm_cache* c, int layer, const void* K, const void* V, co
                       const int32_t* pos, int n);
 
 /*
+ * The step on the input side of the path, fused with svlm_cache_append: the Q/K/V projection of one layer for
+ * the n new tokens, whose epilogue stores keys (rotated at each token's contiguous position, "Contiguous
+ * RoPE" paragraph) and values straight into the tokens' cache slots and hands the queries back:
+ *   [Q | K | V] = X W^T      X bf16 [n][hidden], W bf16 [(q_heads + 2 kv_heads) * head_dim][hidden], rows ordered
+ *                            query heads, key heads, value heads; fp32 accumulation
+ *   Q_out  bf16 [n][q_heads][head_dim], un-rotated (what svlm_attend expects)
+ * token_type / pos as for svlm_cache_append: read by the call with layer 0, which takes the metadata;
+ * calls for layers 1.. of the same tokens follow with the same n (layer-sequential use, layer >= 0 only).
+ * Results equal svlm_cache_append with K, V = the projection's outputs, except that a key is rounded to
+ * bf16 once, after its rotation, instead of before and after.
+ * Requires head_dim 128, hidden a multiple of 64, X, W and Q_out 16-byte aligned.
+ * Errors: SVLM_ERR_ARG, SVLM_ERR_CAPACITY, SVLM_ERR_ORDER as svlm_cache_append.
+ */
+int svlm_qkv_append(svlm_cache* c, int layer, const void* X, const void* W, int hidden, int q_heads,
+                    const uint8_t* token_type, const int32_t* pos, int n, void* Q_out);
+
+/*
  * Evict, compact and re-index, all layers at once ("Streaming-aware KV Cache" and "Contiguous
  * RoPE" paragraphs).  Keeps the n_sink sink tokens, the last text_window text tokens and the last
  * vision_window vision tokens; every retained token's position moves left by the native position

@@ -37,6 +37,7 @@ _lib.svlm_attend.argtypes = [_vp, _i, _vp, _vp, _i, _i, _vp]
 _lib.svlm_decode_step.argtypes = [_vp, _i, _vp, _vp, _vp, _vp, _vp, _i, _vp]
 _lib.svlm_attend_batched.argtypes = [C.POINTER(_vp), _i, _i, _vp, _vp, _i, _i, _vp]
 _lib.svlm_attend_batched_varlen.argtypes = [C.POINTER(_vp), _i, _i, _vp, _vp, C.POINTER(C.c_int32), _i, _vp]
+_lib.svlm_qkv_append.argtypes = [_vp, _i, _vp, _vp, _i, _i, _vp, _vp, _i, _vp]
 _lib.svlm_decode_step_batched.argtypes = [C.POINTER(_vp), _i, _i, _vp, _vp, _vp, _vp, _vp, _i, _vp]
 _lib.svlm_cache_evict_batched.argtypes = [C.POINTER(_vp), _i]
 _lib.svlm_cache_append_host.argtypes = [_vp, _i, _vp, _vp, _vp, _vp, _i]
@@ -124,6 +125,17 @@ class Cache:
         rc = _lib.svlm_cache_append(self._h, layer, _dev_ptr(K, torch.bfloat16), _dev_ptr(V, torch.bfloat16),
                                     _dev_ptr(token_type, torch.uint8), _dev_ptr(pos, torch.int32), n)
         _check(rc, "svlm_cache_append")
+
+    def qkv_append(self, layer, X, W, q_heads, token_type=None, pos=None, Q_out=None):
+        """Projection with the append as its epilogue: X bf16 CUDA [n, hidden], W [(q_heads + 2 kv_heads) * d, hidden];
+        stores the layer's rotated keys and values of the n tokens in the cache and returns Q [n, q_heads, d]."""
+        n, hidden = X.shape
+        if Q_out is None:
+            Q_out = torch.empty(n, q_heads, self.head_dim, dtype=torch.bfloat16, device=X.device)
+        rc = _lib.svlm_qkv_append(self._h, layer, _dev_ptr(X, torch.bfloat16), _dev_ptr(W, torch.bfloat16), hidden, q_heads,
+                                  _dev_ptr(token_type, torch.uint8), _dev_ptr(pos, torch.int32), n, _dev_ptr(Q_out, torch.bfloat16))
+        _check(rc, "svlm_qkv_append")
+        return Q_out
 
     def evict(self):
         _check(_lib.svlm_cache_evict(self._h), "svlm_cache_evict")

@@ -53,6 +53,11 @@ cudaError_t svlm_launch_decode(const SvlmAttendBatch& b, int layer0, int n_layer
                                int q_heads, void* out, int splits, const void* Knew, const void* Vnew, int early_loads,
                                cudaStream_t st);
 
+// Q/K/V projection with the append as its epilogue, head_dim 128 (svlm_qkv_sm100.cu).  tmX, tmW: host copies of
+// the CUtensorMap of X [n][hidden] and W [(q_heads + 2 kv_heads) * 128][hidden] (64 x 128 boxes, 128-byte swizzle).
+cudaError_t svlm_launch_qkv_append(const void* tmX, const void* tmW, const SvlmCacheDev& cd, int layer, int n, int hidden,
+                                   int q_heads, void* Q_out, cudaStream_t st);
+
 // tcgen05/TMEM/TMA chunk prefill, n_q >= 2 (svlm_prefill_sm100.cu)
 bool svlm_prefill_supported(int n_pages, int group);
 cudaError_t svlm_launch_prefill(const SvlmAttendBatch& b, int layer0, int n_layers, const void* Q, const int* q_pos,

@@ -100,13 +100,29 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-int make_tensor_maps(svlm_cache* c) {
+EncodeTiledFn tensor_map_encoder() {
     void* fn = nullptr;
     cudaDriverEntryPointQueryResult qres;
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn ||
         qres != cudaDriverEntryPointSuccess)
-        return SVLM_ERR_CUDA;
-    EncodeTiledFn encode = reinterpret_cast<EncodeTiledFn>(fn);
+        return nullptr;
+    return reinterpret_cast<EncodeTiledFn>(fn);
+}
+
+// Map of a row-major bf16 matrix [rows][cols] with a 64-column x 128-row box and 128-byte swizzle.
+bool encode_matrix_map(EncodeTiledFn encode, CUtensorMap* map, const void* base, long long rows, long long cols) {
+    cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+    cuuint32_t box[2] = {64, 128};
+    cuuint32_t estr[2] = {1, 1};
+    return encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+int make_tensor_maps(svlm_cache* c) {
+    EncodeTiledFn encode = tensor_map_encoder();
+    if (!encode) return SVLM_ERR_CUDA;
     const SvlmCacheDev& d = c->dev;
     alignas(64) CUtensorMap maps[4];
     for (int which = 0; which < 4; ++which) {   // K, V with a whole-page box; K, V with a 32-row box
@@ -367,6 +383,33 @@ int svlm_cache_append(svlm_cache* c, int layer, const void* K, const void* V, co
     }
     svlm_launch_kv_write(c->dev, layer, K, V, n, c->stream);
     SVLM_CUDA(cudaGetLastError());
+    return SVLM_OK;
+}
+
+int svlm_qkv_append(svlm_cache* c, int layer, const void* X, const void* W, int hidden, int q_heads,
+                    const uint8_t* token_type, const int32_t* pos, int n, void* Q_out) {
+    if (!c || !X || !W || !Q_out || n < 1 || layer < 0 || layer >= c->dev.layers) return SVLM_ERR_ARG;
+    if (c->dev.head_dim != 128 || hidden < 64 || hidden % 64 || q_heads < 1 || q_heads % c->dev.kv_heads) return SVLM_ERR_ARG;
+    if (((uintptr_t)X | (uintptr_t)W | (uintptr_t)Q_out) & 15) return SVLM_ERR_ARG;      // TMA and 16-byte stores
+    DeviceGuard guard(c->device);
+    static const EncodeTiledFn encode = tensor_map_encoder();
+    if (!encode) return SVLM_ERR_CUDA;
+    alignas(64) CUtensorMap tmX, tmW;
+    if (!encode_matrix_map(encode, &tmX, X, n, hidden) ||
+        !encode_matrix_map(encode, &tmW, W, (long long)(q_heads + 2 * c->dev.kv_heads) * 128, hidden))
+        return SVLM_ERR_CUDA;
+    c->last_decode_layer = -1;
+    if (layer == 0) {
+        if (!token_type || !pos) return SVLM_ERR_ARG;
+        if (n > c->dev.capacity) return SVLM_ERR_CAPACITY;
+        c->configured_locked = true;
+        svlm_launch_append_meta(c->dev, token_type, pos, n, c->stream);
+        c->appended += n;
+        c->pending_n = n;
+    } else if (n != c->pending_n) {
+        return SVLM_ERR_ORDER;
+    }
+    SVLM_CUDA(svlm_launch_qkv_append(&tmX, &tmW, c->dev, layer, n, hidden, q_heads, Q_out, c->stream));
     return SVLM_OK;
 }
 
