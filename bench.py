@@ -718,6 +718,57 @@ def bench_sweep(args, wl, base, peaks, rank, world, local):
                               roofline=roof, cpu_baseline=None, e2e=None, gpu_launches=None, clocks=None, sweep=rows)))
 
 
+def bench_qkv(args, wl, base, peaks, rank, world, local):
+    """The step on the input side of the path (svlm_qkv_append): the Q/K/V projection of one layer whose epilogue
+    rotates the keys and appends to the cache, timed on the config's head shape with hidden size 3584 for one
+    chunk (n ~ 524) and for a long append (n = 4096), plain calls, CUDA events, weights of different layers in turn
+    (28 x 33 MB > L2)."""
+    import torch
+    from paper_2510_09608_b200 import binding
+    hidden, L = 3584, args.layers or wl.layers
+    n_out = (wl.q_heads + 2 * wl.kv_heads) * wl.head_dim
+    g = torch.Generator(device="cuda").manual_seed(wl.seed)
+    W = (torch.randn(L, n_out, hidden, generator=g, device="cuda") / hidden ** 0.5).to(torch.bfloat16)
+    rows = []
+    for n in (wl.vision_per_chunk + wl.text_max // 2, 4096):
+        cache = binding.Cache(L, wl.kv_heads, wl.head_dim, 0, 0, 0, (n + 127) // 128 * 128)   # every eviction empties it
+        cache.set_rope(wl.rope_mode, wl.rope_base, wl.sections)
+        X = torch.randn(L, n, hidden, generator=g, device="cuda").to(torch.bfloat16)
+        Q = torch.empty(n, wl.q_heads, wl.head_dim, dtype=torch.bfloat16, device="cuda")
+        ty = torch.ones(n, dtype=torch.uint8, device="cuda")
+        times = []
+        for it in range(args.warmup + args.steps):
+            pos = torch.arange(it * n, (it + 1) * n, dtype=torch.int32, device="cuda")
+            if wl.rope_mode:
+                pos = pos[:, None].repeat(1, 3).contiguous()
+            ev = [torch.cuda.Event(enable_timing=True) for _ in range(L + 1)]
+            for l in range(L):
+                if l == 1:
+                    ev[0].record()          # layer 0 also takes the metadata: timed from layer 1 on
+                cache.qkv_append(l, X[l], W[l], wl.q_heads, ty if l == 0 else None, pos if l == 0 else None, Q)
+            ev[1].record()
+            cache.evict()                   # room for the next append
+            torch.cuda.synchronize()
+            if it >= args.warmup:
+                times.append(ev[0].elapsed_time(ev[1]) / (L - 1))
+        assert cache.status() == binding.OK
+        cache.close()
+        ms = statistics.median(times)
+        flops = 2.0 * n * hidden * n_out
+        rows.append(dict(n=n, ms_per_layer=ms, tflops=flops / (ms * 1e-3) / 1e12, frac=flops / (ms * 1e-3) / 1e12 / peaks["bf16_burst"],
+                         ctas=(n + 127) // 128 * (wl.q_heads + 2 * wl.kv_heads)))
+    if rank == 0:
+        d = rows[-1]
+        roof = dict(bound="tensor", kernel="qkv_append", achieved=d["tflops"], peak=peaks["bf16_burst"], unit="TFLOP/s", frac=d["frac"],
+                    traffic=None, algorithmic=2.0 * d["n"] * hidden * n_out, peak_source=peaks["source"] + " (burst bf16)")
+        print(json.dumps(dict(base, metric="layers/s of the Q/K/V projection with append epilogue", unit="layers/s",
+                              value=1e3 / d["ms_per_layer"], ms_per_step=d["ms_per_layer"],
+                              config=dict(workload=f"svlm_qkv_append on the config {args.config} head shape: hidden {hidden} -> "
+                                                   f"{wl.q_heads}+{wl.kv_heads}+{wl.kv_heads} heads of {wl.head_dim}, {L} layers in turn",
+                                          l2="weights of the layers in turn exceed L2; no flush", replicas="independent streams, no collective"),
+                              roofline=roof, cpu_baseline=None, e2e=None, gpu_launches=None, clocks=None, points=rows)))
+
+
 def dataclasses_replace(obj, **kw):
     import dataclasses
     return dataclasses.replace(obj, **kw)
@@ -735,7 +786,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="replay nothing: plain calls in the timed region")
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (smaller case for profiling)")
-    ap.add_argument("--workload", default="step", choices=["step", "overlap", "sweep"],
+    ap.add_argument("--workload", default="step", choices=["step", "overlap", "sweep", "qkv"],
                     help="step: the per-chunk KV-cache step (default); overlap: the whole window re-prefilled every second; "
                          "sweep: the step's latency over the paper's sink / window ablation values")
     args = ap.parse_args()
@@ -789,6 +840,11 @@ def main():
         torch.cuda.synchronize()
 
     peaks = load_peaks()
+    if args.workload == "qkv":
+        bench_qkv(args, sg.workloads()[args.config], base, peaks, rank, world, local)
+        if world > 1:
+            dist.destroy_process_group()
+        return
     if args.workload == "sweep":
         bench_sweep(args, sg.workloads()[args.config], base, peaks, rank, world, local)
         if world > 1:
