@@ -721,7 +721,7 @@ def bench_sweep(args, wl, base, peaks, rank, world, local):
 def bench_qkv(args, wl, base, peaks, rank, world, local):
     """The step on the input side of the path (svlm_qkv_append): the Q/K/V projection of one layer whose epilogue
     rotates the keys and appends to the cache, timed on the config's head shape with hidden size 3584 for one
-    chunk (n ~ 524) and for a long append (n = 4096), plain calls, CUDA events, weights of different layers in turn
+    chunk (n ~ 524) and for a long append (n = 4096), graph replay, CUDA events, weights of different layers in turn
     (28 x 33 MB > L2)."""
     import torch
     from paper_2510_09608_b200 import binding
@@ -736,27 +736,40 @@ def bench_qkv(args, wl, base, peaks, rank, world, local):
         X = torch.randn(L, n, hidden, generator=g, device="cuda").to(torch.bfloat16)
         Q = torch.empty(n, wl.q_heads, wl.head_dim, dtype=torch.bfloat16, device="cuda")
         ty = torch.ones(n, dtype=torch.uint8, device="cuda")
-        times = []
-        for it in range(args.warmup + args.steps):
+        def step(it):
             pos = torch.arange(it * n, (it + 1) * n, dtype=torch.int32, device="cuda")
             if wl.rope_mode:
                 pos = pos[:, None].repeat(1, 3).contiguous()
-            ev = [torch.cuda.Event(enable_timing=True) for _ in range(L + 1)]
             for l in range(L):
-                if l == 1:
-                    ev[0].record()          # layer 0 also takes the metadata: timed from layer 1 on
                 cache.qkv_append(l, X[l], W[l], wl.q_heads, ty if l == 0 else None, pos if l == 0 else None, Q)
-            ev[1].record()
             cache.evict()                   # room for the next append
+
+        step(0)                             # plain once: one-time kernel attributes outside any capture
+        torch.cuda.synchronize()
+        graphs = []
+        cur = torch.cuda.current_stream()
+        for it in range(1, args.warmup + args.steps + 1):   # replayed from graphs: the host's share of a call is not timed
+            gr = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(gr):
+                cache.set_stream(torch.cuda.current_stream())
+                step(it)
+            graphs.append(gr)
+        cache.set_stream(cur)
+        times = []
+        for it, gr in enumerate(graphs):
+            a, b2 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            gr.replay()
+            b2.record()
             torch.cuda.synchronize()
             if it >= args.warmup:
-                times.append(ev[0].elapsed_time(ev[1]) / (L - 1))
+                times.append(a.elapsed_time(b2) / L)   # per layer; the metadata and eviction launches are inside
         assert cache.status() == binding.OK
         cache.close()
         ms = statistics.median(times)
         flops = 2.0 * n * hidden * n_out
         rows.append(dict(n=n, ms_per_layer=ms, tflops=flops / (ms * 1e-3) / 1e12, frac=flops / (ms * 1e-3) / 1e12 / peaks["bf16_burst"],
-                         ctas=(n + 127) // 128 * (wl.q_heads + 2 * wl.kv_heads)))
+                         ctas=(n + 127) // 128 * ((wl.q_heads + 2 * wl.kv_heads + 1) // 2)))
     if rank == 0:
         d = rows[-1]
         roof = dict(bound="tensor", kernel="qkv_append", achieved=d["tflops"], peak=peaks["bf16_burst"], unit="TFLOP/s", frac=d["frac"],

@@ -54,7 +54,7 @@ cudaError_t svlm_launch_decode(const SvlmAttendBatch& b, int layer0, int n_layer
                                cudaStream_t st);
 
 // Q/K/V projection with the append as its epilogue, head_dim 128 (svlm_qkv_sm100.cu).  tmX, tmW: host copies of
-// the CUtensorMap of X [n][hidden] and W [(q_heads + 2 kv_heads) * 128][hidden] (64 x 128 boxes, 128-byte swizzle).
+// the CUtensorMap of X [n][hidden] (64 x 128 box) and W [(q_heads + 2 kv_heads) * 128][hidden] (64 x 256 box), 128-byte swizzle.
 cudaError_t svlm_launch_qkv_append(const void* tmX, const void* tmW, const SvlmCacheDev& cd, int layer, int n, int hidden,
                                    int q_heads, void* Q_out, cudaStream_t st);
 

@@ -5,11 +5,12 @@
 // token's cache slot: K and V never make a round trip through global memory between the GEMM and
 // the cache.
 //
-// A dense contraction, so it runs on the tensor cores: one CTA per 128 x 128 output tile (128 tokens x
-// one head: head_dim is 128, so the rotation partners j and j + 64 of a key sit in the same tile),
-// X and W tiles by TMA (128-byte swizzle) through a 6-stage ring, one thread issuing
-// tcgen05.mma (M128 N128 K16) into a 128-column TMEM accumulator, four epilogue warps reading the
-// accumulator with tcgen05.ld, one row per thread.  Every mbarrier wait is bounded; on expiry the CTA
+// A dense contraction, so it runs on the tensor cores: one CTA per 128 x 256 output tile (128 tokens x
+// two heads: head_dim is 128, so the rotation partners j and j + 64 of a key sit in the same tile; with
+// 128 x 128 tiles the operand stream out of L2, 64 flop per byte, bounded the kernel at ~700 TFLOP/s),
+// X and W tiles by TMA (128-byte swizzle) through a 4-stage ring, one thread issuing
+// tcgen05.mma (M128 N256 K16) into a 256-column TMEM accumulator, four epilogue warps reading the
+// accumulator with tcgen05.ld, one row per thread, one head after the other.  Every mbarrier wait is bounded; on expiry the CTA
 // records SVLM_ERR_TIMEOUT, drains its copies, frees its TMEM and returns.
 #include <cuda.h>
 #include <cuda_bf16.h>
@@ -26,9 +27,10 @@ namespace {
 using namespace svlm_ptx;
 using namespace svlm_tc;
 
-constexpr int QK_STAGES = 6;
+constexpr int QK_STAGES = 4;
 constexpr int QK_BK = 64;                       // k-block: 64 bf16 = one 128-byte swizzle row
-constexpr int QK_TILE = 128 * QK_BK * 2;        // bytes of one operand tile (128 rows)
+constexpr int QK_TILE = 128 * QK_BK * 2;        // bytes of the X tile (128 rows); the W tile (256 rows) is twice that
+constexpr int QK_STAGE = 3 * QK_TILE;
 constexpr int QK_THREADS = 192;                 // warp 0: TMA, warp 1: MMA issue + TMEM, warps 2-5: epilogue
 
 // Out of line: the rare fp64 path of the look-up would otherwise be copied into every unrolled pair.
@@ -48,9 +50,10 @@ qkv_append_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
     constexpr int D = 128, HALF = 64;
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     unsigned char* ring = smem_raw;                                      // [stage][X tile | W tile]
-    QkShared& sh = *reinterpret_cast<QkShared*>(ring + QK_STAGES * 2 * QK_TILE);
+    QkShared& sh = *reinterpret_cast<QkShared*>(ring + QK_STAGES * QK_STAGE);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int head = blockIdx.x;                 // output tile column = head: query heads, key heads, value heads
+    const int head0 = 2 * blockIdx.x;            // the tile's two heads, in the order query heads, key heads, value heads
+    const int n_heads = q_heads + 2 * cd.kv_heads;
     const int m0 = blockIdx.y * 128;             // first token of the tile
     const int n_kb = hidden / QK_BK;
     volatile int* abort_flag = &sh.abort_flag;
@@ -66,7 +69,7 @@ qkv_append_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
         mbar_init_fence();
     }
     if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh.tmem_base)), "r"(128));
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh.tmem_base)), "r"(256));
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
     }
     tc_fence_before();
@@ -80,25 +83,25 @@ qkv_append_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
             for (int kb = 0; kb < n_kb; ++kb) {
                 const int st = kb % QK_STAGES;
                 if (!mbar_wait(&sh.empty[st], ((kb / QK_STAGES) & 1) ^ 1, abort_flag)) break;   // first pass: already free
-                unsigned char* dst = ring + st * 2 * QK_TILE;
-                mbar_expect_tx(&sh.full[st], 2 * QK_TILE);
-                tma_load_2d(dst, &tmX, kb * QK_BK, m0, &sh.full[st]);                 // rows past n read as zeros
-                tma_load_2d(dst + QK_TILE, &tmW, kb * QK_BK, head * D, &sh.full[st]);
+                unsigned char* dst = ring + st * QK_STAGE;
+                mbar_expect_tx(&sh.full[st], QK_STAGE);
+                tma_load_2d(dst, &tmX, kb * QK_BK, m0, &sh.full[st]);                 // rows past the end read as zeros
+                tma_load_2d(dst + QK_TILE, &tmW, kb * QK_BK, head0 * D, &sh.full[st]);
             }
         }
         __syncwarp();
     } else if (warp == 1) {
         // ================= MMA issuer =================
         if (lane == 0) {
-            constexpr unsigned IDESC = make_idesc(128, 128, 0);
+            constexpr unsigned IDESC = make_idesc(128, 256, 0);
             bool ok = true;
             for (int kb = 0; kb < n_kb && ok; ++kb) {
                 const int st = kb % QK_STAGES;
                 ok = mbar_wait(&sh.full[st], (kb / QK_STAGES) & 1, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
-                const unsigned long long da = smem_desc(smem_u32(ring + st * 2 * QK_TILE), 16, 1024);
-                const unsigned long long db = smem_desc(smem_u32(ring + st * 2 * QK_TILE + QK_TILE), 16, 1024);
+                const unsigned long long da = smem_desc(smem_u32(ring + st * QK_STAGE), 16, 1024);
+                const unsigned long long db = smem_desc(smem_u32(ring + st * QK_STAGE + QK_TILE), 16, 1024);
 #pragma unroll
                 for (int ks = 0; ks < QK_BK / 16; ++ks)
                     tc_mma_ss(tmem, da + (unsigned)(ks * 32 >> 4), db + (unsigned)(ks * 32 >> 4), IDESC, (kb | ks) != 0);
@@ -112,17 +115,20 @@ qkv_append_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
         const int quad = warp & 3;                               // the TMEM lane quadrant this warp may read
         const int row = quad * 32 + lane;
         const int i = m0 + row;
-        const unsigned tacc = tmem + ((unsigned)(quad * 32) << 16);
-        const int kv = head - q_heads;                           // < 0: query head; < kv_heads: key head; else value head
-        // where the token lives (key and value tiles): the append's slot, if the append stood
+        // where the token lives (key and value heads): the append's slot, if the append stood
         int slot = -1;
-        if (kv >= 0 && i < n && cd.ctrl->append_n == n) {
+        if (head0 + 1 >= q_heads && i < n && cd.ctrl->append_n == n) {
             const int s = cd.new_slot[i];
             if (cd.slot_gid[s] == cd.ctrl->n_total - n + i) slot = s;
         }
         const bool ok = mbar_wait(&sh.acc_full, 0, abort_flag);
         tc_fence_after();
-        if (ok) {
+#pragma unroll 1
+        for (int hh = 0; hh < 2 && ok; ++hh) {
+            const int head = head0 + hh;
+            if (head >= n_heads) break;                          // odd head count: the last tile is half empty
+            const unsigned tacc = tmem + ((unsigned)(quad * 32) << 16) + hh * D;
+            const int kv = head - q_heads;                       // < 0: query head; < kv_heads: key head; else value head
             if (kv >= 0 && kv < cd.kv_heads) {
                 // key: pairs (j, j + 64), rotated at the slot's current position, 32 pairs at a time
                 uint16_t* dst = cd.K + (((size_t)layer * cd.kv_heads + kv) * cd.n_slots + (slot >= 0 ? slot : 0)) * D;
@@ -191,11 +197,11 @@ qkv_append_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
     }
     if (warp == 1) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(128));
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(256));
     }
 }
 
-constexpr size_t qkv_smem() { return (size_t)QK_STAGES * 2 * QK_TILE + sizeof(QkShared); }
+constexpr size_t qkv_smem() { return (size_t)QK_STAGES * QK_STAGE + sizeof(QkShared); }
 
 }  // namespace
 
@@ -203,7 +209,7 @@ cudaError_t svlm_launch_qkv_append(const void* tmX, const void* tmW, const SvlmC
                                    int q_heads, void* Q_out, cudaStream_t st) {
     cudaError_t e = svlm_allow_smem<qkv_append_kernel>(qkv_smem());
     if (e != cudaSuccess) return e;
-    const dim3 grid(q_heads + 2 * cd.kv_heads, (n + 127) / 128);
+    const dim3 grid((q_heads + 2 * cd.kv_heads + 1) / 2, (n + 127) / 128);
     qkv_append_kernel<<<grid, QK_THREADS, qkv_smem(), st>>>(*static_cast<const CUtensorMap*>(tmX), *static_cast<const CUtensorMap*>(tmW),
                                                              cd, layer, n, hidden, q_heads, static_cast<uint16_t*>(Q_out));
     svlm_count_launch();

@@ -109,11 +109,11 @@ EncodeTiledFn tensor_map_encoder() {
     return reinterpret_cast<EncodeTiledFn>(fn);
 }
 
-// Map of a row-major bf16 matrix [rows][cols] with a 64-column x 128-row box and 128-byte swizzle.
-bool encode_matrix_map(EncodeTiledFn encode, CUtensorMap* map, const void* base, long long rows, long long cols) {
+// Map of a row-major bf16 matrix [rows][cols] with a 64-column x box_rows box and 128-byte swizzle.
+bool encode_matrix_map(EncodeTiledFn encode, CUtensorMap* map, const void* base, long long rows, long long cols, int box_rows) {
     cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
     cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
-    cuuint32_t box[2] = {64, 128};
+    cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
     cuuint32_t estr[2] = {1, 1};
     return encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -395,8 +395,8 @@ int svlm_qkv_append(svlm_cache* c, int layer, const void* X, const void* W, int 
     static const EncodeTiledFn encode = tensor_map_encoder();
     if (!encode) return SVLM_ERR_CUDA;
     alignas(64) CUtensorMap tmX, tmW;
-    if (!encode_matrix_map(encode, &tmX, X, n, hidden) ||
-        !encode_matrix_map(encode, &tmW, W, (long long)(q_heads + 2 * c->dev.kv_heads) * 128, hidden))
+    if (!encode_matrix_map(encode, &tmX, X, n, hidden, 128) ||
+        !encode_matrix_map(encode, &tmW, W, (long long)(q_heads + 2 * c->dev.kv_heads) * 128, hidden, 256))
         return SVLM_ERR_CUDA;
     c->last_decode_layer = -1;
     if (layer == 0) {
