@@ -116,6 +116,15 @@ int svlm_qkv_append(svlm_cache* c, int layer, const void* X, const void* W, int 
                     const uint8_t* token_type, const int32_t* pos, int n, void* Q_out);
 
 /*
+ * The step on the output side of the path: the projection that consumes the attention output,
+ *   Y = A Wo^T      A bf16 [n][in_dim] (svlm_attend's out viewed as [n][q_heads * head_dim]), Wo bf16 [out_dim][in_dim],
+ *                   Y bf16 [n][out_dim]; fp32 accumulation, the same tensor-core kernel as svlm_qkv_append.
+ * Enqueued on the cache's stream (the cache is otherwise untouched).  in_dim a multiple of 64, out_dim a
+ * multiple of 128, pointers 16-byte aligned.  Errors: SVLM_ERR_ARG.
+ */
+int svlm_out_proj(svlm_cache* c, const void* A, const void* Wo, int in_dim, int out_dim, int n, void* Y);
+
+/*
  * Evict, compact and re-index, all layers at once ("Streaming-aware KV Cache" and "Contiguous
  * RoPE" paragraphs).  Keeps the n_sink sink tokens, the last text_window text tokens and the last
  * vision_window vision tokens; every retained token's position moves left by the native position

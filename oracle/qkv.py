@@ -36,6 +36,11 @@ def project(X_bits: np.ndarray, W_bits: np.ndarray, q_heads: int, kv_heads: int,
             Y[:, nq + nk:].reshape(n, kv_heads, head_dim))
 
 
+def out_project(A_bits: np.ndarray, Wo_bits: np.ndarray) -> np.ndarray:
+    """The projection on the output side, y_i = W_o a_i: A bf16 bits [n, in_dim], Wo [out_dim, in_dim] -> fp64 [n, out_dim]."""
+    return widen(A_bits) @ widen(Wo_bits).T
+
+
 def rotate(x: np.ndarray, c: np.ndarray, rope_mode: int, base: float, sections) -> np.ndarray:
     """R(c) x for x [n, heads, d] and integer positions c [n, 3] (1D mode reads column 0)."""
     n, _, d = x.shape

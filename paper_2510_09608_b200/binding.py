@@ -38,6 +38,7 @@ _lib.svlm_decode_step.argtypes = [_vp, _i, _vp, _vp, _vp, _vp, _vp, _i, _vp]
 _lib.svlm_attend_batched.argtypes = [C.POINTER(_vp), _i, _i, _vp, _vp, _i, _i, _vp]
 _lib.svlm_attend_batched_varlen.argtypes = [C.POINTER(_vp), _i, _i, _vp, _vp, C.POINTER(C.c_int32), _i, _vp]
 _lib.svlm_qkv_append.argtypes = [_vp, _i, _vp, _vp, _i, _i, _vp, _vp, _i, _vp]
+_lib.svlm_out_proj.argtypes = [_vp, _vp, _vp, _i, _i, _i, _vp]
 _lib.svlm_decode_step_batched.argtypes = [C.POINTER(_vp), _i, _i, _vp, _vp, _vp, _vp, _vp, _i, _vp]
 _lib.svlm_cache_evict_batched.argtypes = [C.POINTER(_vp), _i]
 _lib.svlm_cache_append_host.argtypes = [_vp, _i, _vp, _vp, _vp, _vp, _i]
@@ -136,6 +137,16 @@ class Cache:
                                   _dev_ptr(token_type, torch.uint8), _dev_ptr(pos, torch.int32), n, _dev_ptr(Q_out, torch.bfloat16))
         _check(rc, "svlm_qkv_append")
         return Q_out
+
+    def out_proj(self, A, Wo, Y=None):
+        """Y = A Wo^T on the cache's stream: A bf16 CUDA [n, in_dim], Wo [out_dim, in_dim] -> Y [n, out_dim]."""
+        n, in_dim = A.shape
+        if Y is None:
+            Y = torch.empty(n, Wo.shape[0], dtype=torch.bfloat16, device=A.device)
+        rc = _lib.svlm_out_proj(self._h, _dev_ptr(A, torch.bfloat16), _dev_ptr(Wo, torch.bfloat16), in_dim, Wo.shape[0], n,
+                                _dev_ptr(Y, torch.bfloat16))
+        _check(rc, "svlm_out_proj")
+        return Y
 
     def evict(self):
         _check(_lib.svlm_cache_evict(self._h), "svlm_cache_evict")

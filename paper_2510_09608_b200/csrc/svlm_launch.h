@@ -55,8 +55,9 @@ cudaError_t svlm_launch_decode(const SvlmAttendBatch& b, int layer0, int n_layer
 
 // Q/K/V projection with the append as its epilogue, head_dim 128 (svlm_qkv_sm100.cu).  tmX, tmW: host copies of
 // the CUtensorMap of X [n][hidden] (64 x 128 box) and W [(q_heads + 2 kv_heads) * 128][hidden] (64 x 256 box), 128-byte swizzle.
+// with_append = false: the plain projection Y = X W^T with q_heads blocks of 128 output columns, all written to Q_out.
 cudaError_t svlm_launch_qkv_append(const void* tmX, const void* tmW, const SvlmCacheDev& cd, int layer, int n, int hidden,
-                                   int q_heads, void* Q_out, cudaStream_t st);
+                                   int q_heads, bool with_append, void* Q_out, cudaStream_t st);
 
 // tcgen05/TMEM/TMA chunk prefill, n_q >= 2 (svlm_prefill_sm100.cu)
 bool svlm_prefill_supported(int n_pages, int group);

@@ -44,16 +44,18 @@ struct QkShared {
     int abort_flag;
 };
 
+// kv_heads_used = cd.kv_heads for the projection with append; 0 turns the kernel into the plain projection
+// Y = X W^T (the output projection after attention): every 128-column block is then a "query head" and goes to Q_out.
 __global__ void __launch_bounds__(QK_THREADS, 1)
 qkv_append_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW, SvlmCacheDev cd,
-                  int layer, int n, int hidden, int q_heads, uint16_t* __restrict__ Q_out) {
+                  int layer, int n, int hidden, int q_heads, int kv_heads_used, uint16_t* __restrict__ Q_out) {
     constexpr int D = 128, HALF = 64;
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     unsigned char* ring = smem_raw;                                      // [stage][X tile | W tile]
     QkShared& sh = *reinterpret_cast<QkShared*>(ring + QK_STAGES * QK_STAGE);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int head0 = 2 * blockIdx.x;            // the tile's two heads, in the order query heads, key heads, value heads
-    const int n_heads = q_heads + 2 * cd.kv_heads;
+    const int n_heads = q_heads + 2 * kv_heads_used;
     const int m0 = blockIdx.y * 128;             // first token of the tile
     const int n_kb = hidden / QK_BK;
     volatile int* abort_flag = &sh.abort_flag;
@@ -206,12 +208,13 @@ constexpr size_t qkv_smem() { return (size_t)QK_STAGES * QK_STAGE + sizeof(QkSha
 }  // namespace
 
 cudaError_t svlm_launch_qkv_append(const void* tmX, const void* tmW, const SvlmCacheDev& cd, int layer, int n, int hidden,
-                                   int q_heads, void* Q_out, cudaStream_t st) {
+                                   int q_heads, bool with_append, void* Q_out, cudaStream_t st) {
     cudaError_t e = svlm_allow_smem<qkv_append_kernel>(qkv_smem());
     if (e != cudaSuccess) return e;
-    const dim3 grid((q_heads + 2 * cd.kv_heads + 1) / 2, (n + 127) / 128);
+    const int kv = with_append ? cd.kv_heads : 0;
+    const dim3 grid((q_heads + 2 * kv + 1) / 2, (n + 127) / 128);
     qkv_append_kernel<<<grid, QK_THREADS, qkv_smem(), st>>>(*static_cast<const CUtensorMap*>(tmX), *static_cast<const CUtensorMap*>(tmW),
-                                                             cd, layer, n, hidden, q_heads, static_cast<uint16_t*>(Q_out));
+                                                             cd, layer, n, hidden, q_heads, kv, static_cast<uint16_t*>(Q_out));
     svlm_count_launch();
     return cudaGetLastError();
 }

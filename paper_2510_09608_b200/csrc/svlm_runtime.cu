@@ -409,7 +409,20 @@ int svlm_qkv_append(svlm_cache* c, int layer, const void* X, const void* W, int 
     } else if (n != c->pending_n) {
         return SVLM_ERR_ORDER;
     }
-    SVLM_CUDA(svlm_launch_qkv_append(&tmX, &tmW, c->dev, layer, n, hidden, q_heads, Q_out, c->stream));
+    SVLM_CUDA(svlm_launch_qkv_append(&tmX, &tmW, c->dev, layer, n, hidden, q_heads, true, Q_out, c->stream));
+    return SVLM_OK;
+}
+
+int svlm_out_proj(svlm_cache* c, const void* A, const void* Wo, int in_dim, int out_dim, int n, void* Y) {
+    if (!c || !A || !Wo || !Y || n < 1 || in_dim < 64 || in_dim % 64 || out_dim < 128 || out_dim % 128) return SVLM_ERR_ARG;
+    if (((uintptr_t)A | (uintptr_t)Wo | (uintptr_t)Y) & 15) return SVLM_ERR_ARG;
+    DeviceGuard guard(c->device);
+    static const EncodeTiledFn encode = tensor_map_encoder();
+    if (!encode) return SVLM_ERR_CUDA;
+    alignas(64) CUtensorMap tmA, tmW;
+    if (!encode_matrix_map(encode, &tmA, A, n, in_dim, 128) || !encode_matrix_map(encode, &tmW, Wo, out_dim, in_dim, 256))
+        return SVLM_ERR_CUDA;
+    SVLM_CUDA(svlm_launch_qkv_append(&tmA, &tmW, c->dev, 0, n, in_dim, out_dim / 128, false, Y, c->stream));
     return SVLM_OK;
 }
 

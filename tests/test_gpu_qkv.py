@@ -77,6 +77,25 @@ def test_projection_with_append_full_size_layer():
     assert n >= 512
 
 
+@pytest.mark.parametrize("n,in_dim,out_dim", [(70, 128, 384), (300, 192, 128), (524, 3584, 3584)])
+def test_output_projection(n, in_dim, out_dim):
+    """svlm_out_proj against the fp64 product: ragged row tiles, an odd number of 128-column blocks, the full layer."""
+    from harness import bits_to_dev, dev_to_f64
+    from oracle import qkv
+    from paper_2510_09608_b200 import binding
+    rng = np.random.default_rng(n)
+    A = qkv.to_bf16_bits(rng.standard_normal((n, in_dim)))
+    W = qkv.to_bf16_bits(rng.standard_normal((out_dim, in_dim)) / np.sqrt(in_dim))
+    c = binding.Cache(1, 1, 128, 4, 64, 16, 256)
+    Y = dev_to_f64(c.out_proj(bits_to_dev(A), bits_to_dev(W)))
+    want = qkv.out_project(A, W)
+    assert c.status() == binding.OK
+    assert np.all(np.abs(Y - want) <= 2.0 ** -8 * np.abs(want) + 1e-5 * np.sqrt(in_dim))
+    with pytest.raises(binding.SvlmError) as e:
+        c.out_proj(bits_to_dev(A), bits_to_dev(W[:out_dim - 64]))        # out_dim must be a multiple of 128
+    assert e.value.status == binding.ERR_ARG
+
+
 def test_projection_argument_errors():
     from paper_2510_09608_b200 import binding
     c = binding.Cache(1, 2, 128, 4, 64, 16, 256)

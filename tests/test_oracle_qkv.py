@@ -25,6 +25,20 @@ def test_selector_weights_copy_input_columns():
     assert np.array_equal(V.reshape(n, -1), Y[:, (qh + kh) * d:])
 
 
+def test_output_projection_selector_and_loop():
+    rng = np.random.default_rng(5)
+    A, W = _bits(rng, (4, 12)), _bits(rng, (7, 12))
+    Y = qkv.out_project(A, W)
+    Af, Wf = qkv.widen(A), qkv.widen(W)
+    for i in range(4):
+        for o in range(7):
+            want = sum(float(Af[i, k]) * float(Wf[o, k]) for k in range(12))
+            assert abs(Y[i, o] - want) <= 1e-12 * max(1.0, abs(want))
+    S = np.zeros((5, 12))
+    S[np.arange(5), [3, 0, 11, 7, 7]] = 1.0
+    assert np.array_equal(qkv.out_project(A, qkv.to_bf16_bits(S)), Af[:, [3, 0, 11, 7, 7]])
+
+
 def test_projection_is_the_triple_loop():
     rng = np.random.default_rng(2)
     n, hidden, qh, kh, d = 3, 16, 2, 1, 4
