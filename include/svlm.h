@@ -158,6 +158,8 @@ int svlm_attend(svlm_cache* c, int layer, const void* Q, const int32_t* q_pos, i
  *   token_type  uint8 [1], pos int32 [1] or [3]: the metadata is taken by the call with layer 0;
  *               calls for layers 1.. of the same token follow and may pass null token_type (pos is
  *               still needed: it is the query's position).
+ * layer -1 takes all layers of the token in ONE launch, for callers that hold every layer's inputs at once (an
+ * attention-only stack, a benchmark): K, V are [layers][kv_heads][head_dim], Q and out [layers][q_heads][head_dim].
  * At most 8 query heads per KV head.  Consecutive calls for different layers of the same token
  * overlap on the GPU (the next layer's cache pages are fetched while the previous layer finishes);
  * K, V, Q and everything else produced by earlier work in the stream are read only after that work

@@ -461,10 +461,10 @@ int svlm_attend(svlm_cache* c, int layer, const void* Q, const int32_t* q_pos, i
 
 int svlm_decode_step(svlm_cache* c, int layer, const void* K, const void* V, const uint8_t* token_type,
                      const int32_t* pos, const void* Q, int q_heads, void* out) {
-    if (!c || !K || !V || !pos || !Q || !out || layer < 0 || layer >= c->dev.layers || q_heads < 1) return SVLM_ERR_ARG;
+    if (!c || !K || !V || !pos || !Q || !out || layer < -1 || layer >= c->dev.layers || q_heads < 1) return SVLM_ERR_ARG;
     if (q_heads % c->dev.kv_heads || q_heads / c->dev.kv_heads > 8) return SVLM_ERR_ARG;
     DeviceGuard guard(c->device);
-    if (layer == 0) {
+    if (layer <= 0) {
         if (!token_type) return SVLM_ERR_ARG;
         c->configured_locked = true;
         c->last_decode_layer = -1;

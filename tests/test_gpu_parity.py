@@ -128,6 +128,33 @@ def test_eight_query_heads_per_kv_head_and_all_layers_decode():
         assert_close(s.attend(2, all_layers=True))
 
 
+def test_fused_decode_step_all_layers_in_one_launch():
+    """svlm_decode_step with layer -1: one token's append and attention for all layers at once."""
+    from harness import SideBySide, assert_close, bits_to_dev, dev_to_f64
+    from paper_2510_09608_b200 import binding
+    wl = dataclasses.replace(_wl(2), layers=3, n_sink=16, vision_window=256, text_window=32, frames=1, grid_h=8, grid_w=8)
+    s = SideBySide(wl)
+    for _ in range(4):
+        s.append_chunk()
+        s.evict()
+    for step in range(3):
+        gids, types, pos = s.stream.next_decode_token()
+        K = np.stack([s.stream.k(l, gids)[0] for l in range(wl.layers)])
+        V = np.stack([s.stream.v(l, gids)[0] for l in range(wl.layers)])
+        Q = np.stack([s.stream.q(l, gids)[0] for l in range(wl.layers)])
+        out = dev_to_f64(s.cache.decode_step(-1, bits_to_dev(K), bits_to_dev(V), torch.from_numpy(types).cuda(),
+                                             torch.from_numpy(np.ascontiguousarray(pos)).cuda(), bits_to_dev(Q)))
+        assert s.cache.status() == binding.OK
+        s.ref.append(None, None, types, pos)
+        s.last = (gids, types, pos)
+        for l in range(wl.layers):
+            s._give_values_to_ref(l)
+            assert_close(s._stats(out[l][None], s.ref.attend(l, Q[l][None], pos)))
+    s.check_metadata()
+    for l in range(wl.layers):
+        s.check_kv(l)
+
+
 def test_batched_streams_match_single_calls():
     from harness import SideBySide, bits_to_dev, dev_to_f64
     from paper_2510_09608_b200 import binding
