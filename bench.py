@@ -770,6 +770,26 @@ def bench_qkv(args, wl, base, peaks, rank, world, local):
         flops = 2.0 * n * hidden * n_out
         rows.append(dict(n=n, ms_per_layer=ms, tflops=flops / (ms * 1e-3) / 1e12, frac=flops / (ms * 1e-3) / 1e12 / peaks["bf16_burst"],
                          ctas=(n + 127) // 128 * ((wl.q_heads + 2 * wl.kv_heads + 1) // 2)))
+    # decode-time projections (a few tokens): the bandwidth kernel behind svlm_out_proj, weights of the layers in turn
+    cache = binding.Cache(1, wl.kv_heads, wl.head_dim, 0, 0, 0, 128)
+    small = []
+    for n in (1, 16):
+        x = torch.randn(n, hidden, generator=g, device="cuda").to(torch.bfloat16)
+        y = torch.empty(n, n_out, dtype=torch.bfloat16, device="cuda")
+        ts = []
+        for it in range(args.warmup + args.steps):
+            a, b2 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for l in range(L):
+                cache.out_proj(x, W[l], y)
+            b2.record()
+            torch.cuda.synchronize()
+            if it >= args.warmup:
+                ts.append(a.elapsed_time(b2) / L)
+        ms = statistics.median(ts)
+        wbytes = n_out * hidden * 2
+        small.append(dict(n=n, ms_per_layer=ms, gbs=wbytes / (ms * 1e-3) / 1e9, frac_hbm=wbytes / (ms * 1e-3) / 1e9 / peaks["hbm"]))
+    cache.close()
     if rank == 0:
         d = rows[-1]
         roof = dict(bound="tensor", kernel="qkv_append", achieved=d["tflops"], peak=peaks["bf16_burst"], unit="TFLOP/s", frac=d["frac"],
@@ -779,7 +799,8 @@ def bench_qkv(args, wl, base, peaks, rank, world, local):
                               config=dict(workload=f"svlm_qkv_append on the config {args.config} head shape: hidden {hidden} -> "
                                                    f"{wl.q_heads}+{wl.kv_heads}+{wl.kv_heads} heads of {wl.head_dim}, {L} layers in turn",
                                           l2="weights of the layers in turn exceed L2; no flush", replicas="independent streams, no collective"),
-                              roofline=roof, cpu_baseline=None, e2e=None, gpu_launches=None, clocks=None, points=rows)))
+                              roofline=roof, cpu_baseline=None, e2e=None, gpu_launches=None, clocks=None, points=rows,
+                              decode_projection=small)))
 
 
 def dataclasses_replace(obj, **kw):

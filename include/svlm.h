@@ -119,6 +119,8 @@ int svlm_qkv_append(svlm_cache* c, int layer, const void* X, const void* W, int 
  * The step on the output side of the path: the projection that consumes the attention output,
  *   Y = A Wo^T      A bf16 [n][in_dim] (svlm_attend's out viewed as [n][q_heads * head_dim]), Wo bf16 [out_dim][in_dim],
  *                   Y bf16 [n][out_dim]; fp32 accumulation, the same tensor-core kernel as svlm_qkv_append.
+ * Up to 16 rows (decode) take a bandwidth kernel that reads Wo once instead.  The same call serves the input
+ * side of a decode step: [q | k | v] = svlm_out_proj(x, W_qkv) is laid out as svlm_decode_step's Q, K and V.
  * Enqueued on the cache's stream (the cache is otherwise untouched).  in_dim a multiple of 64, out_dim a
  * multiple of 128, pointers 16-byte aligned.  Errors: SVLM_ERR_ARG.
  */

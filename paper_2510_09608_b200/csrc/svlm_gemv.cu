@@ -1,0 +1,105 @@
+// Projections of a few tokens at a time (decode): Y = X W^T for n <= 16 rows of X.  With so few rows the
+// work is reading W once, so this is a bandwidth kernel, not a tensor-core one: a warp owns output rows
+// (one row of W each, 16-byte loads, several in flight per lane), multiplies them with all n token vectors
+// held in shared memory, accumulates in fp32 and reduces with shuffles.  It serves svlm_out_proj for small
+// n, on both sides of the decode step: [q | k | v] = W_qkv x before svlm_decode_step, W_o a after it.
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include "svlm_dev.h"
+#include "svlm_launch.h"
+
+namespace {
+
+constexpr int GV_THREADS = 256;
+// 16-byte chunks of a W row in flight per lane: the fewer token vectors share the registers, the more loads
+template <int NX> __host__ __device__ constexpr int gv_unroll() { return NX == 1 ? 16 : (NX <= 4 ? 8 : 4); }
+
+template <int NX>
+__global__ void __launch_bounds__(GV_THREADS) gemv_kernel(const uint16_t* __restrict__ X, const uint16_t* __restrict__ W,
+                                                         uint16_t* __restrict__ Y, int n, int in_dim, int out_dim) {
+    constexpr int GV_UNROLL = gv_unroll<NX>();
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    uint4* sx = reinterpret_cast<uint4*>(smem_raw);            // [NX][in_dim / 8] chunks of 8 bf16; rows >= n are zero
+    const int chunks = in_dim / 8;
+    for (int i = threadIdx.x; i < NX * chunks; i += GV_THREADS) {
+        const int t = i / chunks;
+        sx[i] = t < n ? *reinterpret_cast<const uint4*>(X + (size_t)t * in_dim + (size_t)(i % chunks) * 8) : make_uint4(0, 0, 0, 0);
+    }
+    __syncthreads();
+    const int lane = threadIdx.x & 31;
+    const int warp = blockIdx.x * (GV_THREADS / 32) + (threadIdx.x >> 5), n_warps = gridDim.x * (GV_THREADS / 32);
+    for (int row = warp; row < out_dim; row += n_warps) {
+        const uint4* wrow = reinterpret_cast<const uint4*>(W + (size_t)row * in_dim);
+        float acc[NX];
+#pragma unroll
+        for (int t = 0; t < NX; ++t) acc[t] = 0.f;
+        for (int c0 = lane; c0 < chunks; c0 += 32 * GV_UNROLL) {
+            uint4 w[GV_UNROLL];
+#pragma unroll
+            for (int u = 0; u < GV_UNROLL; ++u) {
+                const int c = c0 + 32 * u;
+                w[u] = c < chunks ? __ldg(wrow + c) : make_uint4(0, 0, 0, 0);
+            }
+#pragma unroll
+            for (int u = 0; u < GV_UNROLL; ++u) {
+                const int c = c0 + 32 * u;
+                if (c >= chunks) continue;
+                const __nv_bfloat162* wp = reinterpret_cast<const __nv_bfloat162*>(&w[u]);
+                float2 wf[4];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) wf[q] = __bfloat1622float2(wp[q]);
+#pragma unroll
+                for (int t = 0; t < NX; ++t) {
+                    const uint4 xv = sx[t * chunks + c];
+                    const __nv_bfloat162* xp = reinterpret_cast<const __nv_bfloat162*>(&xv);
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const float2 xf = __bfloat1622float2(xp[q]);
+                        acc[t] = fmaf(wf[q].x, xf.x, acc[t]);
+                        acc[t] = fmaf(wf[q].y, xf.y, acc[t]);
+                    }
+                }
+            }
+        }
+#pragma unroll
+        for (int t = 0; t < NX; ++t) {
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) acc[t] += __shfl_xor_sync(0xffffffffu, acc[t], o);
+        }
+        if (lane == 0) {
+#pragma unroll
+            for (int t = 0; t < NX; ++t)
+                if (t < n) Y[(size_t)t * out_dim + row] = __bfloat16_as_ushort(__float2bfloat16_rn(acc[t]));
+        }
+    }
+}
+
+template <int NX>
+cudaError_t launch(const uint16_t* X, const uint16_t* W, uint16_t* Y, int n, int in_dim, int out_dim, cudaStream_t st) {
+    const size_t smem = (size_t)NX * in_dim * 2;
+    cudaError_t e = svlm_allow_smem<gemv_kernel<NX>>(smem);
+    if (e != cudaSuccess) return e;
+    const int rows_per_block = GV_THREADS / 32;
+    int blocks = (out_dim + rows_per_block - 1) / rows_per_block;
+    if (blocks > 2 * 148) blocks = 2 * 148;         // two resident blocks per SM, each warp walks a few rows
+    gemv_kernel<NX><<<blocks, GV_THREADS, smem, st>>>(X, W, Y, n, in_dim, out_dim);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+bool svlm_gemv_supported(int n, int in_dim) { return n >= 1 && n <= 16 && in_dim % 8 == 0 && (size_t)16 * in_dim * 2 <= 200 * 1024; }
+
+cudaError_t svlm_launch_gemv(const void* X, const void* W, void* Y, int n, int in_dim, int out_dim, cudaStream_t st) {
+    const uint16_t* x = static_cast<const uint16_t*>(X);
+    const uint16_t* w = static_cast<const uint16_t*>(W);
+    uint16_t* y = static_cast<uint16_t*>(Y);
+    cudaError_t e;
+    if (n == 1) e = launch<1>(x, w, y, n, in_dim, out_dim, st);
+    else if (n <= 4) e = launch<4>(x, w, y, n, in_dim, out_dim, st);
+    else if (n <= 8) e = launch<8>(x, w, y, n, in_dim, out_dim, st);
+    else e = launch<16>(x, w, y, n, in_dim, out_dim, st);
+    svlm_count_launch();
+    return e;
+}

@@ -59,6 +59,10 @@ cudaError_t svlm_launch_decode(const SvlmAttendBatch& b, int layer0, int n_layer
 cudaError_t svlm_launch_qkv_append(const void* tmX, const void* tmW, const SvlmCacheDev& cd, int layer, int n, int hidden,
                                    int q_heads, bool with_append, void* Q_out, cudaStream_t st);
 
+// Y = X W^T for a few rows of X (decode-time projections), a bandwidth kernel (svlm_gemv.cu)
+bool svlm_gemv_supported(int n, int in_dim);
+cudaError_t svlm_launch_gemv(const void* X, const void* W, void* Y, int n, int in_dim, int out_dim, cudaStream_t st);
+
 // tcgen05/TMEM/TMA chunk prefill, n_q >= 2 (svlm_prefill_sm100.cu)
 bool svlm_prefill_supported(int n_pages, int group);
 cudaError_t svlm_launch_prefill(const SvlmAttendBatch& b, int layer0, int n_layers, const void* Q, const int* q_pos,

@@ -417,6 +417,10 @@ int svlm_out_proj(svlm_cache* c, const void* A, const void* Wo, int in_dim, int 
     if (!c || !A || !Wo || !Y || n < 1 || in_dim < 64 || in_dim % 64 || out_dim < 128 || out_dim % 128) return SVLM_ERR_ARG;
     if (((uintptr_t)A | (uintptr_t)Wo | (uintptr_t)Y) & 15) return SVLM_ERR_ARG;
     DeviceGuard guard(c->device);
+    if (svlm_gemv_supported(n, in_dim)) {      // a few tokens (decode): reading Wo once is all the work
+        SVLM_CUDA(svlm_launch_gemv(A, Wo, Y, n, in_dim, out_dim, c->stream));
+        return SVLM_OK;
+    }
     static const EncodeTiledFn encode = tensor_map_encoder();
     if (!encode) return SVLM_ERR_CUDA;
     alignas(64) CUtensorMap tmA, tmW;

@@ -77,7 +77,8 @@ def test_projection_with_append_full_size_layer():
     assert n >= 512
 
 
-@pytest.mark.parametrize("n,in_dim,out_dim", [(70, 128, 384), (300, 192, 128), (524, 3584, 3584)])
+@pytest.mark.parametrize("n,in_dim,out_dim", [(70, 128, 384), (300, 192, 128), (524, 3584, 3584),
+                                              (1, 3584, 4608), (3, 192, 128), (8, 3584, 3584), (16, 1024, 640)])
 def test_output_projection(n, in_dim, out_dim):
     """svlm_out_proj against the fp64 product: ragged row tiles, an odd number of 128-column blocks, the full layer."""
     from harness import bits_to_dev, dev_to_f64
@@ -94,6 +95,39 @@ def test_output_projection(n, in_dim, out_dim):
     with pytest.raises(binding.SvlmError) as e:
         c.out_proj(bits_to_dev(A), bits_to_dev(W[:out_dim - 64]))        # out_dim must be a multiple of 128
     assert e.value.status == binding.ERR_ARG
+
+
+def test_decode_step_fed_by_the_projection():
+    """One generated token the way a decoder layer runs it: [q | k | v] = W_qkv x through svlm_out_proj (the
+    bandwidth kernel for a single row), then svlm_decode_step on the three slices; against the fp64 projection
+    rounded to bf16 and the cache checker."""
+    from harness import SideBySide, assert_close, bits_to_dev, dev_to_f64
+    from oracle import qkv
+    from paper_2510_09608_b200 import streamgen as sg
+    wl = dataclasses.replace(sg.workloads()[2], layers=2, n_sink=16, vision_window=256, text_window=32, frames=1, grid_h=8, grid_w=8)
+    hidden, d = 256, wl.head_dim
+    rng = np.random.default_rng(21)
+    s = SideBySide(wl)
+    for _ in range(3):
+        s.append_chunk()
+        s.evict()
+    nq, nk = wl.q_heads * d, wl.kv_heads * d
+    for step in range(2):
+        gids, types, pos = s.stream.next_decode_token()
+        ty, ps = torch.from_numpy(types).cuda(), torch.from_numpy(np.ascontiguousarray(pos)).cuda()
+        s.ref.append(None, None, types, pos)
+        for l in range(wl.layers):
+            x = qkv.to_bf16_bits(rng.standard_normal((1, hidden)))
+            W = qkv.to_bf16_bits(rng.standard_normal((nq + 2 * nk, hidden)) / np.sqrt(hidden))
+            y = s.cache.out_proj(bits_to_dev(x), bits_to_dev(W))                       # [1, (Hq + 2 Hkv) d]
+            Q, K, V = y[:, :nq].view(1, wl.q_heads, d), y[:, nq:nq + nk].view(1, wl.kv_heads, d), y[:, nq + nk:].view(1, wl.kv_heads, d)
+            out = dev_to_f64(s.cache.decode_step(l, K.contiguous(), V.contiguous(), ty if l == 0 else None, ps, Q.contiguous()))
+            Q64, K64, V64 = qkv.project(x, W, wl.q_heads, wl.kv_heads, d)
+            old = s.ref.query()["gids"][:-1]
+            s.ref.set_kv(l, old, s.stream.k(l, old), s.stream.v(l, old)) if step == 0 else None
+            s.ref.set_kv(l, gids, qkv.to_bf16_bits(K64), qkv.to_bf16_bits(V64))
+            assert_close(s._stats(out, s.ref.attend(l, qkv.to_bf16_bits(Q64), pos)), tight=False)
+    s.check_metadata()
 
 
 def test_projection_argument_errors():
