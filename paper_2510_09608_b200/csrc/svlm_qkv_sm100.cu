@@ -38,6 +38,18 @@ __device__ __noinline__ float2 rope_cs_call(const float2* tab, int pair, long lo
     return svlm_rope_cs(tab, 64, pair, c, theta);
 }
 
+// The table look-up without the fp64 path: |c| < 2^24 (see svlm_rope.cuh).
+__device__ __forceinline__ float2 rope_cs_fast(const float2* __restrict__ tab, int pair, int c) {
+    const unsigned u = (unsigned)(c < 0 ? -c : c);
+    float2 r = __ldg(tab + (size_t)(u & 255u) * 64 + pair);
+    if (u >> 8) {
+        r = svlm_cmul(r, __ldg(tab + (size_t)(256 + ((u >> 8) & 255u)) * 64 + pair));
+        if (u >> 16) r = svlm_cmul(r, __ldg(tab + (size_t)(512 + (u >> 16)) * 64 + pair));
+    }
+    if (c < 0) r.y = -r.y;
+    return r;
+}
+
 struct QkShared {
     unsigned long long full[QK_STAGES], empty[QK_STAGES], acc_full;
     unsigned tmem_base;
@@ -123,6 +135,24 @@ qkv_append_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
             const int s = cd.new_slot[i];
             if (cd.slot_gid[s] == cd.ctrl->n_total - n + i) slot = s;
         }
+        // A tile with key heads: the token's 64 rotation factors are looked up into registers now, while the
+        // tensor pipe is still busy with the tile (64 dependent-latency look-ups after it took longer than the GEMM).
+        const float2* tab = reinterpret_cast<const float2*>(cd.rope_tab);
+        float2 cs[HALF];
+        bool have_cs = false;
+        int cpos[3] = {0, 0, 0};
+        if (slot >= 0 && head0 < q_heads + kv_heads_used) {
+            cpos[0] = cd.slot_c[slot]; cpos[1] = cd.slot_c[cd.n_slots + slot]; cpos[2] = cd.slot_c[2 * cd.n_slots + slot];
+            const int lim = 1 << 24;
+            have_cs = cpos[0] > -lim && cpos[0] < lim && cpos[1] > -lim && cpos[1] < lim && cpos[2] > -lim && cpos[2] < lim;
+            if (have_cs) {
+#pragma unroll
+                for (int pair = 0; pair < HALF; ++pair) {
+                    const int axis = cd.rope_mode == 0 ? 0 : (pair < cd.sec_t ? 0 : (pair < cd.sec_th ? 1 : 2));
+                    cs[pair] = rope_cs_fast(tab, pair, axis == 0 ? cpos[0] : (axis == 1 ? cpos[1] : cpos[2]));
+                }
+            }
+        }
         const bool ok = mbar_wait(&sh.acc_full, 0, abort_flag);
         tc_fence_after();
 #pragma unroll 1
@@ -134,23 +164,26 @@ qkv_append_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
             if (kv >= 0 && kv < cd.kv_heads) {
                 // key: pairs (j, j + 64), rotated at the slot's current position, 32 pairs at a time
                 uint16_t* dst = cd.K + (((size_t)layer * cd.kv_heads + kv) * cd.n_slots + (slot >= 0 ? slot : 0)) * D;
-                const float2* tab = reinterpret_cast<const float2*>(cd.rope_tab);
-#pragma unroll 1
+#pragma unroll
                 for (int c32 = 0; c32 < 2; ++c32) {
                     float lo[32], hi[32];
                     tmem_ld32(tacc + c32 * 32, lo);
                     tmem_ld32(tacc + HALF + c32 * 32, hi);
                     tmem_wait_ld();
                     if (slot >= 0) {
-                        const int cpos[3] = {cd.slot_c[slot], cd.slot_c[cd.n_slots + slot], cd.slot_c[2 * cd.n_slots + slot]};
 #pragma unroll
                         for (int k = 0; k < 32; ++k) {
                             const int pair = c32 * 32 + k;
-                            const int axis = cd.rope_mode == 0 ? 0 : (pair < cd.sec_t ? 0 : (pair < cd.sec_th ? 1 : 2));
-                            const float2 cs = rope_cs_call(tab, pair, axis == 0 ? cpos[0] : (axis == 1 ? cpos[1] : cpos[2]), cd.theta[pair]);
+                            float2 f;
+                            if (have_cs) {
+                                f = cs[pair];
+                            } else {   // a position beyond the table's range (native positions of a very long stream)
+                                const int axis = cd.rope_mode == 0 ? 0 : (pair < cd.sec_t ? 0 : (pair < cd.sec_th ? 1 : 2));
+                                f = rope_cs_call(tab, pair, axis == 0 ? cpos[0] : (axis == 1 ? cpos[1] : cpos[2]), cd.theta[pair]);
+                            }
                             const float x = lo[k], y = hi[k];
-                            lo[k] = x * cs.x - y * cs.y;
-                            hi[k] = y * cs.x + x * cs.y;
+                            lo[k] = x * f.x - y * f.y;
+                            hi[k] = y * f.x + x * f.y;
                         }
 #pragma unroll
                         for (int k = 0; k < 4; ++k) {
