@@ -110,6 +110,7 @@ decode_kernel(SvlmAttendBatch b, int layer0, int n_layers, const uint16_t* __res
     unsigned char* ring = reinterpret_cast<unsigned char*>(
         (reinterpret_cast<uintptr_t>(smem_raw) + sizeof(DecShared) + 1023) & ~(uintptr_t)1023);
     uint16_t* s_q = reinterpret_cast<uint16_t*>(ring + DEC_STAGES * STAGE_BYTES);   // [8][D] bf16
+    uint16_t* s_new = s_q + 8 * D;       // fused step: the new token's rotated key [D], then its value [D]
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int g = lane >> 2, t = lane & 3;
@@ -212,6 +213,16 @@ decode_kernel(SvlmAttendBatch b, int layer0, int n_layers, const uint16_t* __res
             }
             constexpr int HSTEP = (DEC_CWARPS * 32) / HALF, HN = (8 + HSTEP - 1) / HSTEP;   // heads per thread
             uint16_t qx[HN], qy[HN];
+            // fused step: the new token's key and value rows come in with the query (same round trip); the key is
+            // rotated with the query's factors (same token, same position) and both wait in shared memory for the
+            // warp whose sub-tile holds the token's slot
+            const bool prep_new = new_slot >= 0 && threadIdx.x < HALF;
+            uint16_t kx = 0, ky = 0, vx = 0, vy = 0;
+            if (prep_new) {
+                const size_t noff = ((size_t)prob * b.kv_heads + hk) * D;
+                kx = Knew[noff + pair]; ky = Knew[noff + pair + HALF];
+                vx = Vnew[noff + pair]; vy = Vnew[noff + pair + HALF];
+            }
 #pragma unroll
             for (int k = 0; k < HN; ++k) {      // all loads first: one round trip
                 const int h = threadIdx.x / HALF + k * HSTEP;
@@ -227,6 +238,13 @@ decode_kernel(SvlmAttendBatch b, int layer0, int n_layers, const uint16_t* __res
                 const float y = h < G ? __bfloat162float(__ushort_as_bfloat16(qy[k])) : 0.f;
                 s_q[h * D + pair] = __bfloat16_as_ushort(__float2bfloat16_rn(x * cs.x - y * cs.y));
                 s_q[h * D + pair + HALF] = __bfloat16_as_ushort(__float2bfloat16_rn(y * cs.x + x * cs.y));
+            }
+            if (prep_new) {
+                const float x = __bfloat162float(__ushort_as_bfloat16(kx)), y = __bfloat162float(__ushort_as_bfloat16(ky));
+                s_new[pair] = __bfloat16_as_ushort(__float2bfloat16_rn(x * cs.x - y * cs.y));
+                s_new[pair + HALF] = __bfloat16_as_ushort(__float2bfloat16_rn(y * cs.x + x * cs.y));
+                s_new[D + pair] = vx;
+                s_new[D + pair + HALF] = vy;
             }
         }
         asm volatile("bar.sync 1, %0;" ::"n"(DEC_CWARPS * 32));   // consumer warps only
@@ -263,19 +281,11 @@ decode_kernel(SvlmAttendBatch b, int layer0, int n_layers, const uint16_t* __res
                 // fused append: rotate the new key at its position, put key and value into the
                 // shared-memory row and into the cache
                 const int r = new_slot & 31;
-                const uint16_t* ksrc = Knew + ((size_t)prob * b.kv_heads + hk) * D;
-                const uint16_t* vsrc = Vnew + ((size_t)prob * b.kv_heads + hk) * D;
                 uint16_t* kdst = const_cast<uint16_t*>(vw.K) + (head_row0 + new_slot) * D;
                 uint16_t* vdst = const_cast<uint16_t*>(vw.V) + (head_row0 + new_slot) * D;
                 for (int pair = lane; pair < HALF; pair += 32) {
-                    const int axis = b.rope_mode == 0 ? 0 : (pair < b.sec_t ? 0 : (pair < b.sec_th ? 1 : 2));
-                    const long long c = __ldcg(vw.slot_c + (size_t)axis * b.n_slots + new_slot);
-                    const float2 cs = svlm_rope_cs(tab, HALF, pair, c, b.theta[pair]);
-                    const float x = __bfloat162float(__ushort_as_bfloat16(ksrc[pair]));
-                    const float y = __bfloat162float(__ushort_as_bfloat16(ksrc[pair + HALF]));
-                    const uint16_t klo = __bfloat16_as_ushort(__float2bfloat16_rn(x * cs.x - y * cs.y));
-                    const uint16_t khi = __bfloat16_as_ushort(__float2bfloat16_rn(y * cs.x + x * cs.y));
-                    const uint16_t vlo = vsrc[pair], vhi = vsrc[pair + HALF];
+                    const uint16_t klo = s_new[pair], khi = s_new[pair + HALF];
+                    const uint16_t vlo = s_new[D + pair], vhi = s_new[D + pair + HALF];
                     kdst[pair] = klo; kdst[pair + HALF] = khi;
                     vdst[pair] = vlo; vdst[pair + HALF] = vhi;
                     const int e0 = pair, e1 = pair + HALF;
@@ -506,7 +516,7 @@ decode_kernel(SvlmAttendBatch b, int layer0, int n_layers, const uint16_t* __res
 
 template <int D>
 constexpr size_t decode_smem() {
-    return sizeof(DecShared) + 1024 + (size_t)DEC_STAGES * 2 * SUB * D * 2 + 8 * D * 2;
+    return sizeof(DecShared) + 1024 + (size_t)DEC_STAGES * 2 * SUB * D * 2 + 8 * D * 2 + 2 * D * 2;
 }
 
 }  // namespace
