@@ -142,10 +142,133 @@ __device__ void rebuild_tiles(const SvlmCacheDev& cd, int sink_fill, const long 
 }
 
 // ---------------------------------------------------------------------------------------------
+// Append of ONE token (every decode step): the same bookkeeping as the general kernel below without its
+// block-wide scans, and with the list of active pages edited instead of rebuilt: a single token changes
+// one entry (the last page of its ring, or of the sinks, grows by one slot) or adds one (a page opens),
+// which shifts the entries behind it.  The old entries are fetched while the control block is still on
+// its way, so the kernel is two dependent round trips (control block, then page table or free stack)
+// instead of six.  Returns false, having done nothing, when the list is longer than the block.
+__device__ __forceinline__ bool append_one_body(const SvlmCacheDev& cd, const unsigned char* types, const int* pos) {
+    __shared__ int s_state;       // 0: go on; 1: append dropped (capacity)
+    SvlmCtrl* ctrl = cd.ctrl;
+    const int tid = threadIdx.x;
+    SvlmTile old;                 // entry `tid` of the present list (garbage beyond its end; never used then)
+    if (tid < cd.n_pages) old = cd.tiles[tid];
+    const int n_tiles0 = ctrl->n_tiles;
+    if (n_tiles0 > (int)blockDim.x) return false;          // uniform: every thread reads the same word
+    const long long n_total0 = ctrl->n_total;
+    const int ty = types[0] ? 1 : 0;
+    const long long ord = ctrl->n_type[ty];
+    const long long cursor0 = ctrl->cursor;
+    const long long shift = cd.contiguous ? ctrl->shift_total : 0;
+    const long long ring_n0[2] = {ctrl->ring_n[0], ctrl->ring_n[1]};
+    const long long ring_lo0[2] = {ctrl->ring_lo[0], ctrl->ring_lo[1]};
+    const int sink_fill0 = ctrl->sink_fill;
+    const int n_stored0 = ctrl->n_stored;
+    const int free_top0 = ctrl->free_top;
+    long long p[3];
+    if (cd.rope_mode == 0) { p[0] = p[1] = p[2] = pos[0]; }
+    else { p[0] = pos[0]; p[1] = pos[1]; p[2] = pos[2]; }
+
+    const long long gid = n_total0;
+    const bool is_sink = cd.sink_any ? (gid < cd.n_sink) : (ty == 0 && ord < cd.n_sink);
+    const long long u = ring_n0[ty];                       // the token's ring ordinal if it is not a sink
+    const bool new_page = !is_sink && (u % SVLM_PAGE) == 0;
+    // the list as it is: sink pages, text ring pages, vision ring pages
+    const int ns0 = (sink_fill0 + SVLM_PAGE - 1) / SVLM_PAGE;
+    int cnt0[2];
+    for (int t = 0; t < 2; ++t)
+        cnt0[t] = ring_n0[t] > ring_lo0[t] ? (int)((ring_n0[t] - 1) / SVLM_PAGE - ring_lo0[t] / SVLM_PAGE + 1) : 0;
+    // the entry the token lands in: position in the OLD list if it exists there, else where it is inserted
+    bool adds;              // a new entry appears
+    int at;                 // old index of the entry that grows, or new index of the entry that appears
+    if (is_sink) {
+        adds = (sink_fill0 % SVLM_PAGE) == 0;
+        at = adds ? ns0 : ns0 - 1;
+    } else {
+        const int cnt1 = (int)(u / SVLM_PAGE - ring_lo0[ty] / SVLM_PAGE + 1);
+        adds = cnt1 != cnt0[ty];
+        at = ns0 + (ty ? cnt0[0] : 0) + (adds ? cnt0[ty] : cnt0[ty] - 1);
+    }
+    if (tid == 0) {
+        const bool ok = (n_stored0 + 1 <= cd.capacity) && (!new_page || free_top0 >= 1) &&
+                        (!is_sink || sink_fill0 + 1 <= cd.n_sink_pages * SVLM_PAGE);
+        s_state = ok ? 0 : 1;
+        if (!ok) {
+            ctrl->append_n = 0;
+            if (ctrl->status == 0) ctrl->status = -2;   // SVLM_ERR_CAPACITY
+        }
+    }
+    __syncthreads();                                    // also: every old entry is in registers
+    if (s_state) return true;
+
+    // entries behind an inserted one move up by one; the one that grows is rewritten by its owner
+    if (tid < n_tiles0) {
+        if (adds && tid >= at) cd.tiles[tid + 1] = old;
+        if (!adds && tid == at) {
+            old.hi += 1;
+            old.max_gid = gid;
+            cd.tiles[tid] = old;
+        }
+    }
+    if (tid == 0) {
+        int slot, page;
+        if (is_sink) {
+            slot = (int)(cd.sink_any ? gid : ord);
+            page = slot / SVLM_PAGE;
+        } else {
+            const int pt = (int)(u / SVLM_PAGE) & (cd.pt_size - 1);
+            if (new_page) {
+                page = cd.free_stack[free_top0 - 1];
+                cd.page_table[ty][pt] = page;
+                ctrl->free_top = free_top0 - 1;
+            } else {
+                page = cd.page_table[ty][pt];
+            }
+            slot = page * SVLM_PAGE + (int)(u % SVLM_PAGE);
+        }
+        if (adds) {
+            SvlmTile tl;
+            tl.page = page;
+            tl.lo = slot % SVLM_PAGE;
+            tl.hi = tl.lo + 1;
+            tl.pad = 0;
+            tl.min_gid = tl.max_gid = gid;
+            cd.tiles[at] = tl;
+            ctrl->n_tiles = n_tiles0 + 1;
+        }
+        const long long top = max(p[0], max(p[1], p[2])) + 1;
+        cd.slot_gid[slot] = gid;
+        cd.slot_type[slot] = (unsigned char)ty;
+        cd.slot_a[slot] = (int)max(0ll, top - cursor0);
+        cd.slot_delta[slot] = 0;
+        cd.new_slot[0] = slot;
+        for (int k = 0; k < 3; ++k) {
+            const int c = (int)(p[k] - shift);
+            cd.slot_c[k * cd.n_slots + slot] = c;
+            cd.new_c[k] = c;
+        }
+        ctrl->n_total = n_total0 + 1;
+        ctrl->n_type[ty] = ord + 1;
+        ctrl->cursor = max(cursor0, top);
+        if (is_sink) {
+            ctrl->sink_cnt[ty] += 1;
+            ctrl->sink_fill = sink_fill0 + 1;
+        } else {
+            ctrl->ring_n[ty] = u + 1;
+        }
+        ctrl->n_stored = n_stored0 + 1;
+        ctrl->append_n = 1;
+    }
+    return true;
+}
+
+// ---------------------------------------------------------------------------------------------
 // Append: stream ordinal, per-type ordinal, cursor advance a = max(0, max(p)+1 - cursor),
 // contiguous position c = p - shift_total, and the storage slot of each of the n new tokens.
 __device__ __forceinline__ void append_meta_body(const SvlmCacheDev& cd, const unsigned char* types, const int* pos,
                                                  int n) {
+    if (n == 1 && append_one_body(cd, types, pos)) return;
     __shared__ int wbuf[META_WARPS];
     __shared__ long long wbuf64[META_WARPS];
     __shared__ int s_cnt[3];     // text tokens; sink tokens of type TEXT / VISION in this append

@@ -261,6 +261,47 @@ def test_batched_chunk_prefill_with_chunks_of_different_lengths():
     assert e.value.status == binding.ERR_ARG
 
 
+@pytest.mark.parametrize("sink_any", [False, True])
+def test_one_token_appends_equal_bulk_appends(sink_any):
+    """The single-token append (its own short kernel path, which edits the list of active pages) against the
+    general append of the same tokens in one call and against the checker: mixed types, sinks filling up, pages
+    opening in the sink area and in both rings, evictions in between; metadata bit-exact at every check."""
+    import oracle
+    from paper_2510_09608_b200 import binding
+    rng = np.random.default_rng(7 + sink_any)
+    args = (1, 1, 64, 150, 200, 140, 1024)       # layers, kv heads, d, sinks, vision window, text window, capacity
+    one, bulk = binding.Cache(*args), binding.Cache(*args)
+    ref = oracle.Oracle(1, 1, 64, 150, 200, 140, sink_any_type=sink_any)
+    for c in (one, bulk):
+        c.set_policy(sink_any, True)
+    z = lambda n: torch.zeros(n, 1, 64, dtype=torch.bfloat16, device="cuda")  # noqa: E731
+    nxt = 0
+    for rnd in range(12):
+        n = int(rng.integers(40, 300))
+        types = (rng.random(n) < (0.7 if rnd % 3 else 0.2)).astype(np.uint8)        # mostly vision, sometimes mostly text
+        pos = np.arange(nxt, nxt + n, dtype=np.int32)
+        nxt += n
+        ty, ps = torch.from_numpy(types).cuda(), torch.from_numpy(pos).cuda()
+        bulk.append(0, z(n), z(n), ty, ps)
+        for i in range(n):
+            one.append(0, z(1), z(1), ty[i:i + 1], ps[i:i + 1])
+        ref.append(None, None, types, pos)
+        for check in (False, True):
+            a, b, w = one.query(), bulk.query(), ref.query()
+            assert one.status() == binding.OK and bulk.status() == binding.OK
+            for k in ("gids", "types", "pos"):
+                assert np.array_equal(a[k], b[k]) and np.array_equal(a[k], w[k]), (rnd, check, k)
+            assert a["shift_total"] == b["shift_total"] == w["shift_total"]
+            if not check:
+                one.evict(); bulk.evict(); ref.evict()
+    # a single-token append beyond the capacity is dropped on the device and reported
+    small = binding.Cache(1, 1, 64, 4, 8, 8, 16)
+    for i in range(17):
+        small.append(0, z(1), z(1), torch.zeros(1, dtype=torch.uint8, device="cuda"), torch.full((1,), i, dtype=torch.int32, device="cuda"))
+        assert small.status() == (binding.OK if i < 16 else binding.ERR_CAPACITY)
+    assert len(small.query()["gids"]) == 16
+
+
 def test_errors_and_capacity():
     from paper_2510_09608_b200 import binding
     with pytest.raises(binding.SvlmError):
