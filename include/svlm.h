@@ -213,7 +213,9 @@ int svlm_cache_evict_batched(svlm_cache* const* caches, int n_caches);
  * Host-buffer variants: the same operations with K, V, token_type, pos / Q, q_pos, out in HOST
  * memory (pinned memory makes the copies asynchronous).  The library stages them through device
  * buffers it owns (grown on demand, which synchronises once).  svlm_attend_host returns after the
- * result has arrived in out_host (it synchronises the stream).
+ * result has arrived in out_host (it synchronises the stream).  For all layers of a chunk (layer -1, n_q >= 2)
+ * svlm_attend_host runs the layers as a pipeline on two copy streams of its own beside the cache's stream, so
+ * that one layer's copies hide behind another layer's attention; pinned host buffers are needed for that.
  */
 int svlm_cache_append_host(svlm_cache* c, int layer, const void* K_host, const void* V_host,
                            const uint8_t* token_type_host, const int32_t* pos_host, int n);

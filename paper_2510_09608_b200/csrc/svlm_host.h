@@ -24,4 +24,8 @@ struct svlm_cache {
     // staging for the *_host entry points
     void* stage = nullptr;
     size_t stage_bytes = 0;
+    // copy streams and per-layer events of the pipelined host-buffer chunk prefill (created on first use)
+    cudaStream_t copy_in = nullptr, copy_out = nullptr;
+    cudaEvent_t ev_start = nullptr;
+    std::vector<cudaEvent_t> ev_in, ev_done;
 };

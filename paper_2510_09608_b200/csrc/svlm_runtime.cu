@@ -328,6 +328,11 @@ void svlm_cache_destroy(svlm_cache* c) {
     cudaStreamSynchronize(c->stream);
     for (void* p : c->allocs) cudaFree(p);
     if (c->stage) cudaFree(c->stage);
+    if (c->copy_in) { cudaStreamSynchronize(c->copy_in); cudaStreamDestroy(c->copy_in); }
+    if (c->copy_out) { cudaStreamSynchronize(c->copy_out); cudaStreamDestroy(c->copy_out); }
+    if (c->ev_start) cudaEventDestroy(c->ev_start);
+    for (cudaEvent_t e : c->ev_in) cudaEventDestroy(e);
+    for (cudaEvent_t e : c->ev_done) cudaEventDestroy(e);
     delete c;
 }
 
@@ -578,6 +583,47 @@ int svlm_attend_host(svlm_cache* c, int layer, const void* Q_host, const int32_t
     int rc = ensure_stage(c, 2 * q_bytes + pos_bytes);
     if (rc != SVLM_OK) return rc;
     char* s = static_cast<char*>(c->stage);
+    if (layer < 0 && nl > 1 && n_q >= 2) {
+        // All layers of a chunk: the layers' queries go up, are attended and their outputs come down as a
+        // pipeline over three streams, so that the copies of one layer hide behind the attention of another.
+        if (!c->copy_in) {
+            SVLM_CUDA(cudaStreamCreateWithFlags(&c->copy_in, cudaStreamNonBlocking));
+            SVLM_CUDA(cudaStreamCreateWithFlags(&c->copy_out, cudaStreamNonBlocking));
+            SVLM_CUDA(cudaEventCreateWithFlags(&c->ev_start, cudaEventDisableTiming));
+        }
+        while ((int)c->ev_in.size() < nl) {
+            cudaEvent_t a = nullptr, b = nullptr;
+            SVLM_CUDA(cudaEventCreateWithFlags(&a, cudaEventDisableTiming));
+            c->ev_in.push_back(a);
+            SVLM_CUDA(cudaEventCreateWithFlags(&b, cudaEventDisableTiming));
+            c->ev_done.push_back(b);
+        }
+        const size_t layer_bytes = (size_t)n_q * q_heads * c->dev.head_dim * 2;
+        const size_t pos_n = (size_t)n_q * (c->dev.rope_mode == SVLM_ROPE_1D ? 1 : 3) * sizeof(int32_t);
+        // the staging buffer may still be in use by earlier work on the cache's stream
+        SVLM_CUDA(cudaEventRecord(c->ev_start, c->stream));
+        SVLM_CUDA(cudaStreamWaitEvent(c->copy_in, c->ev_start, 0));
+        SVLM_CUDA(cudaMemcpyAsync(s + 2 * q_bytes, q_pos_host, pos_n, cudaMemcpyHostToDevice, c->stream));
+        for (int l = 0; l < nl; ++l) {
+            SVLM_CUDA(cudaMemcpyAsync(s + l * layer_bytes, static_cast<const char*>(Q_host) + l * layer_bytes, layer_bytes,
+                                      cudaMemcpyHostToDevice, c->copy_in));
+            SVLM_CUDA(cudaEventRecord(c->ev_in[l], c->copy_in));
+        }
+        for (int l = 0; l < nl; ++l) {
+            SVLM_CUDA(cudaStreamWaitEvent(c->stream, c->ev_in[l], 0));
+            rc = svlm_attend(c, l, s + l * layer_bytes, reinterpret_cast<const int32_t*>(s + 2 * q_bytes), n_q, q_heads,
+                             s + q_bytes + l * layer_bytes);
+            if (rc != SVLM_OK) break;
+            SVLM_CUDA(cudaEventRecord(c->ev_done[l], c->stream));
+            SVLM_CUDA(cudaStreamWaitEvent(c->copy_out, c->ev_done[l], 0));
+            SVLM_CUDA(cudaMemcpyAsync(static_cast<char*>(out_host) + l * layer_bytes, s + q_bytes + l * layer_bytes, layer_bytes,
+                                      cudaMemcpyDeviceToHost, c->copy_out));
+        }
+        SVLM_CUDA(cudaStreamSynchronize(c->copy_in));
+        SVLM_CUDA(cudaStreamSynchronize(c->stream));
+        SVLM_CUDA(cudaStreamSynchronize(c->copy_out));
+        return rc;
+    }
     SVLM_CUDA(cudaMemcpyAsync(s, Q_host, (size_t)nl * n_q * q_heads * c->dev.head_dim * 2, cudaMemcpyHostToDevice,
                               c->stream));
     SVLM_CUDA(cudaMemcpyAsync(s + 2 * q_bytes, q_pos_host,

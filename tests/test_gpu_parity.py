@@ -302,6 +302,38 @@ def test_one_token_appends_equal_bulk_appends(sink_any):
     assert len(small.query()["gids"]) == 16
 
 
+def test_host_buffer_entry_points_equal_the_device_ones():
+    """svlm_cache_append_host / svlm_attend_host (pinned host buffers, all layers per call; the chunk prefill runs as a
+    copy/attend pipeline over the layers) against the device-pointer calls on a twin cache: same bits out."""
+    from harness import bits_to_dev
+    from paper_2510_09608_b200 import binding, streamgen as sg
+    wl = dataclasses.replace(_wl(2), layers=3, n_sink=16, vision_window=256, text_window=32, frames=2, grid_h=8, grid_w=8)
+    stream = sg.Stream(wl, 0)
+    mk = lambda: binding.Cache(wl.layers, wl.kv_heads, wl.head_dim, wl.n_sink, wl.vision_window, wl.text_window, wl.capacity)  # noqa: E731
+    dev, host = mk(), mk()
+    for c in (dev, host):
+        c.set_rope(wl.rope_mode, wl.rope_base, wl.sections)
+    pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()  # noqa: E731
+    for step in range(4):
+        for gids, types, pos in [stream.next_chunk()] + [stream.next_decode_token() for _ in range(2)]:
+            K = np.stack([stream.k(l, gids) for l in range(wl.layers)])
+            V = np.stack([stream.v(l, gids) for l in range(wl.layers)])
+            Q = np.stack([stream.q(l, gids) for l in range(wl.layers)])
+            ty, ps = torch.from_numpy(types), torch.from_numpy(np.ascontiguousarray(pos))
+            dev.append(-1, bits_to_dev(K), bits_to_dev(V), ty.cuda(), ps.cuda())
+            host.append_host(-1, pin(K.view(np.int16)), pin(V.view(np.int16)), ty.pin_memory(), ps.pin_memory())
+            if len(gids) > 1:
+                dev.evict()
+                host.evict()
+            want = dev.attend(-1, bits_to_dev(Q), ps.cuda())
+            got = torch.empty(Q.shape, dtype=torch.int16).pin_memory()
+            host.attend_host(-1, pin(Q.view(np.int16)), ps.pin_memory(), got)
+            assert host.status() == binding.OK
+            assert np.array_equal(got.numpy().view(np.uint16), want.view(torch.int16).cpu().numpy().view(np.uint16)), step
+    a, b = dev.query(), host.query()
+    assert np.array_equal(a["gids"], b["gids"]) and np.array_equal(a["pos"], b["pos"])
+
+
 def test_errors_and_capacity():
     from paper_2510_09608_b200 import binding
     with pytest.raises(binding.SvlmError):
