@@ -231,9 +231,8 @@ def run_step_host(cache, wl, inp):
     cache.append_host(-1, inp.h["K"], inp.h["V"], inp.h["types"], inp.h["pos"])
     cache.evict()
     cache.attend_host(-1, inp.h["Q"], inp.h["pos"], inp.h["out"])
-    for d in inp.hdec:
-        cache.append_host(-1, d["K"], d["V"], d["types"], d["pos"])
-        cache.attend_host(-1, d["Q"], d["pos"], d["out"])
+    for d in inp.hdec:      # one generated token: all layers' append and attention fused, one call
+        cache.decode_step_host(-1, d["K"], d["V"], d["types"], d["pos"], d["Q"], d["out"])
 
 
 def fill_to_steady_state(cache, wl, stream):
@@ -1038,7 +1037,7 @@ def main():
         e2e_s = max_over_ranks(e2e_s, world)
         e2e = dict(value=whole_job_value(world, frames_per_step, e2e_s * 1e3), unit="frames/s", ms_per_step=e2e_s * 1e3,
                    h2d_bytes_per_step=hin[1].h2d_bytes(), d2h_bytes_per_step=hin[1].d2h_bytes(),
-                   api="svlm_cache_append_host / svlm_attend_host, all layers per call, pinned host buffers")
+                   api="svlm_cache_append_host / svlm_attend_host / svlm_decode_step_host, all layers per call, pinned host buffers")
 
     elapsed_ms = max_over_ranks(elapsed_ms, world)
     ms_per_step = elapsed_ms / args.steps

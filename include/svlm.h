@@ -221,6 +221,9 @@ int svlm_cache_append_host(svlm_cache* c, int layer, const void* K_host, const v
                            const uint8_t* token_type_host, const int32_t* pos_host, int n);
 int svlm_attend_host(svlm_cache* c, int layer, const void* Q_host, const int32_t* q_pos_host, int n_q, int q_heads,
                      void* out_host);
+/* svlm_decode_step with host buffers (layer -1: all layers of the token in one launch); returns with out_host filled. */
+int svlm_decode_step_host(svlm_cache* c, int layer, const void* K_host, const void* V_host, const uint8_t* token_type_host,
+                          const int32_t* pos_host, const void* Q_host, int q_heads, void* out_host);
 
 /*
  * Decode attention (one query token, as svlm_attend with n_q == 1 and layer >= 0) for callers that

@@ -43,6 +43,7 @@ _lib.svlm_decode_step_batched.argtypes = [C.POINTER(_vp), _i, _i, _vp, _vp, _vp,
 _lib.svlm_cache_evict_batched.argtypes = [C.POINTER(_vp), _i]
 _lib.svlm_cache_append_host.argtypes = [_vp, _i, _vp, _vp, _vp, _vp, _i]
 _lib.svlm_attend_host.argtypes = [_vp, _i, _vp, _vp, _i, _i, _vp]
+_lib.svlm_decode_step_host.argtypes = [_vp, _i, _vp, _vp, _vp, _vp, _vp, _i, _vp]
 _lib.svlm_attend_decode_noalloc.argtypes = [_vp, _i, _vp, _vp, _i, _vp]
 _lib.svlm_cache_query.argtypes = [_vp, _i64p, _vp, _vp, _vp, _i64p]
 _lib.svlm_cache_read_kv.argtypes = [_vp, _i, _vp, _vp]
@@ -194,6 +195,13 @@ class Cache:
         n_q, q_heads = Q.shape[-3], Q.shape[-2]
         rc = _lib.svlm_attend_host(self._h, layer, _host_ptr(Q), _host_ptr(q_pos), n_q, q_heads, _host_ptr(out))
         _check(rc, "svlm_attend_host")
+        return out
+
+    def decode_step_host(self, layer, K, V, token_type, pos, Q, out):
+        """decode_step with HOST buffers: K, V [layers, 1, kv_heads, d] (layer -1) or [1, kv_heads, d]; fills `out`."""
+        rc = _lib.svlm_decode_step_host(self._h, layer, _host_ptr(K), _host_ptr(V), _host_ptr(token_type), _host_ptr(pos),
+                                        _host_ptr(Q), Q.shape[-2], _host_ptr(out))
+        _check(rc, "svlm_decode_step_host")
         return out
 
     def query(self):

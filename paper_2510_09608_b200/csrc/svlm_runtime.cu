@@ -637,6 +637,33 @@ int svlm_attend_host(svlm_cache* c, int layer, const void* Q_host, const int32_t
     return SVLM_OK;
 }
 
+int svlm_decode_step_host(svlm_cache* c, int layer, const void* K_host, const void* V_host, const uint8_t* token_type_host,
+                          const int32_t* pos_host, const void* Q_host, int q_heads, void* out_host) {
+    if (!c || !K_host || !V_host || !pos_host || !Q_host || !out_host || q_heads < 1 || layer < -1 || layer >= c->dev.layers)
+        return SVLM_ERR_ARG;
+    if (layer <= 0 && !token_type_host) return SVLM_ERR_ARG;
+    DeviceGuard guard(c->device);
+    const int nl = layer < 0 ? c->dev.layers : 1;
+    auto up = [](size_t x) { return (x + 255) / 256 * 256; };
+    const size_t kv_bytes = (size_t)nl * c->dev.kv_heads * c->dev.head_dim * 2, q_bytes = (size_t)nl * q_heads * c->dev.head_dim * 2;
+    const size_t pos_bytes = (c->dev.rope_mode == SVLM_ROPE_1D ? 1 : 3) * sizeof(int32_t);
+    const size_t oK = 0, oV = up(kv_bytes), oQ = oV + up(kv_bytes), oO = oQ + up(q_bytes), oP = oO + up(q_bytes), oT = oP + 256;
+    int rc = ensure_stage(c, oT + 256);
+    if (rc != SVLM_OK) return rc;
+    char* s = static_cast<char*>(c->stage);
+    SVLM_CUDA(cudaMemcpyAsync(s + oK, K_host, kv_bytes, cudaMemcpyHostToDevice, c->stream));
+    SVLM_CUDA(cudaMemcpyAsync(s + oV, V_host, kv_bytes, cudaMemcpyHostToDevice, c->stream));
+    SVLM_CUDA(cudaMemcpyAsync(s + oQ, Q_host, q_bytes, cudaMemcpyHostToDevice, c->stream));
+    SVLM_CUDA(cudaMemcpyAsync(s + oP, pos_host, pos_bytes, cudaMemcpyHostToDevice, c->stream));
+    if (layer <= 0) SVLM_CUDA(cudaMemcpyAsync(s + oT, token_type_host, 1, cudaMemcpyHostToDevice, c->stream));
+    rc = svlm_decode_step(c, layer, s + oK, s + oV, reinterpret_cast<const uint8_t*>(s + oT), reinterpret_cast<const int32_t*>(s + oP),
+                          s + oQ, q_heads, s + oO);
+    if (rc != SVLM_OK) return rc;
+    SVLM_CUDA(cudaMemcpyAsync(out_host, s + oO, q_bytes, cudaMemcpyDeviceToHost, c->stream));
+    SVLM_CUDA(cudaStreamSynchronize(c->stream));
+    return SVLM_OK;
+}
+
 // Host mirror of the stored tokens in stream order: (gid, slot) pairs sorted by gid.
 static int snapshot(svlm_cache* c, std::vector<std::pair<long long, int>>& order, SvlmCtrl& ctrl) {
     const SvlmCacheDev& d = c->dev;

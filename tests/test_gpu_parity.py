@@ -320,14 +320,18 @@ def test_host_buffer_entry_points_equal_the_device_ones():
             V = np.stack([stream.v(l, gids) for l in range(wl.layers)])
             Q = np.stack([stream.q(l, gids) for l in range(wl.layers)])
             ty, ps = torch.from_numpy(types), torch.from_numpy(np.ascontiguousarray(pos))
-            dev.append(-1, bits_to_dev(K), bits_to_dev(V), ty.cuda(), ps.cuda())
-            host.append_host(-1, pin(K.view(np.int16)), pin(V.view(np.int16)), ty.pin_memory(), ps.pin_memory())
+            got = torch.empty(Q.shape, dtype=torch.int16).pin_memory()
             if len(gids) > 1:
+                dev.append(-1, bits_to_dev(K), bits_to_dev(V), ty.cuda(), ps.cuda())
+                host.append_host(-1, pin(K.view(np.int16)), pin(V.view(np.int16)), ty.pin_memory(), ps.pin_memory())
                 dev.evict()
                 host.evict()
-            want = dev.attend(-1, bits_to_dev(Q), ps.cuda())
-            got = torch.empty(Q.shape, dtype=torch.int16).pin_memory()
-            host.attend_host(-1, pin(Q.view(np.int16)), ps.pin_memory(), got)
+                want = dev.attend(-1, bits_to_dev(Q), ps.cuda())
+                host.attend_host(-1, pin(Q.view(np.int16)), ps.pin_memory(), got)
+            else:       # a generated token: the fused step, device pointers against host buffers
+                want = dev.decode_step(-1, bits_to_dev(K[:, 0]), bits_to_dev(V[:, 0]), ty.cuda(), ps.cuda(), bits_to_dev(Q[:, 0]))[:, None]
+                host.decode_step_host(-1, pin(K.view(np.int16)), pin(V.view(np.int16)), ty.pin_memory(), ps.pin_memory(),
+                                      pin(Q.view(np.int16)), got)
             assert host.status() == binding.OK
             assert np.array_equal(got.numpy().view(np.uint16), want.view(torch.int16).cpu().numpy().view(np.uint16)), step
     a, b = dev.query(), host.query()
