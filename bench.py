@@ -540,7 +540,7 @@ def bench_multi_stream(args, wl, base, config, peaks, rank, world, local):
     kd = kernels[dominant]
     roofline = dict(bound="tensor" if dominant == "prefill" else "hbm", kernel=dominant, achieved=kd["achieved"],
                     peak=kd["peak"], unit=kd["unit"], frac=kd["frac"], traffic=None,
-                    algorithmic=(flops_b if dominant == "prefill" else kv_bytes_layer if dominant == "decode" else evict_bytes),
+                    algorithmic=(flops if dominant == "prefill" else kv_bytes_layer if dominant == "decode" else evict_bytes),
                     peak_source=peaks["source"] + (" (burst bf16)" if dominant == "prefill" else " (copy)"))
     if rank == 0:
         config = dict(config, replicas="independent streams, no collective",
@@ -1009,7 +1009,7 @@ def main():
         traffic = None          # the counters were taken on the config-3 shape
     roofline = dict(bound="tensor" if dominant == "prefill" else "hbm", kernel=dominant, achieved=kd["achieved"],
                     peak=kd["peak"], unit=kd["unit"], frac=kd["frac"], traffic=traffic,
-                    algorithmic=(flops if dominant == "prefill" else kv_bytes_layer if dominant == "decode" else evict_bytes),
+                    algorithmic=(flops_b if dominant == "prefill" else kv_bytes_layer if dominant == "decode" else evict_bytes),
                     peak_source=peaks["source"] + (" (burst bf16)" if dominant == "prefill" else " (copy)"))
 
     # ---- extra: one token's decode of ALL layers in one launch (svlm_decode_step with layer -1) -----
