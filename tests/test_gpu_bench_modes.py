@@ -26,6 +26,7 @@ def _run(*args):
     (["--config", "5", "--layers", "2", "--steps", "2", "--warmup", "3"], ["kernels"]),
     (["--workload", "overlap", "--layers", "2", "--steps", "3", "--warmup", "3"], ["kernels"]),
     (["--workload", "qkv", "--layers", "2", "--steps", "2", "--warmup", "3"], ["points", "decode_projection"]),
+    (["--workload", "sweep", "--layers", "1"], ["sweep"]),
 ])
 def test_bench_workloads_print_one_json_line(args, keys):
     d = _run(*args)
