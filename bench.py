@@ -802,6 +802,75 @@ def bench_qkv(args, wl, base, peaks, rank, world, local):
                               decode_projection=small)))
 
 
+def bench_drift(args, wl, base, peaks, rank, world, local):
+    """The whole stream of the config (3600 one-second chunks = one hour for config 3), every chunk timed: the paper's
+    claim is a per-chunk latency that stays flat however long the stream runs (Section 3.3).  Plain calls, one CUDA
+    event pair per chunk; key, value and query VALUES are drawn once and reused (they do not influence the time),
+    token types and positions follow the stream.  Reports the drift: ratio of the medians of the last and the first
+    5 % of the chunks after the windows have filled, and the slope of a straight-line fit."""
+    import torch
+    from paper_2510_09608_b200 import binding
+    L = args.layers or wl.layers
+    w = dataclasses_replace(wl, layers=L)
+    chunks = args.chunks or w.chunks
+    stream = sg.Stream(w, rank)
+    cache = binding.Cache(L, w.kv_heads, w.head_dim, w.n_sink, w.vision_window, w.text_window, w.capacity)
+    cache.set_rope(w.rope_mode, w.rope_base, w.sections)
+    fill = fill_to_steady_state(cache, w, stream)
+    cache.evict()
+    g = torch.Generator(device="cuda").manual_seed(w.seed)
+    nmax = w.max_chunk_tokens
+    rnd = lambda *shape: torch.randn(*shape, generator=g, device="cuda").to(torch.bfloat16)  # noqa: E731
+    K, V, Q = rnd(L, nmax, w.kv_heads, w.head_dim), rnd(L, nmax, w.kv_heads, w.head_dim), rnd(L, nmax, w.q_heads, w.head_dim)
+    out = torch.empty_like(Q)
+    k1, v1, q1 = rnd(L, 1, w.kv_heads, w.head_dim), rnd(L, 1, w.kv_heads, w.head_dim), rnd(L, 1, w.q_heads, w.head_dim)
+    o1 = torch.empty_like(q1)
+    text1 = torch.zeros(1, dtype=torch.uint8, device="cuda")
+    sampler = ClockSampler(local)
+    sampler.start()
+    evs = []
+    for i in range(chunks - fill):
+        gids, types, pos = stream.next_chunk()
+        n = len(gids)
+        ty, ps = torch.from_numpy(types).cuda(), torch.from_numpy(np.ascontiguousarray(pos)).cuda()
+        dec = [torch.from_numpy(np.ascontiguousarray(stream.next_decode_token()[2])).cuda() for _ in range(w.decode_steps)]
+        a, b2 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        cache.append(0, K[0, :n], V[0, :n], ty, ps)
+        cache.evict()
+        cache.attend(0, Q[0, :n], ps, out[0, :n])
+        for l in range(1, L):
+            cache.append(l, K[l, :n], V[l, :n])
+            cache.attend(l, Q[l, :n], ps, out[l, :n])
+        for p1 in dec:
+            for l in range(L):
+                cache.decode_step(l, k1[l], v1[l], text1 if l == 0 else None, p1, q1[l], o1[l])
+        b2.record()
+        evs.append((a, b2))
+        if i % 64 == 63:
+            torch.cuda.synchronize()      # keep the host from running far ahead of the device
+    torch.cuda.synchronize()
+    clocks = sampler.finish()
+    assert cache.status() == binding.OK
+    meta = cache.query()
+    lat = np.array([a.elapsed_time(b2) for a, b2 in evs])
+    k5 = max(1, len(lat) // 20)
+    first, last = float(np.median(lat[:k5])), float(np.median(lat[-k5:]))
+    slope = float(np.polyfit(np.arange(len(lat)), lat, 1)[0]) * 1000.0
+    if rank == 0:
+        print(json.dumps(dict(base, value=w.frames / (float(np.median(lat)) * 1e-3), ms_per_step=float(np.median(lat)), steps=len(lat),
+                              config=dict(workload=f"config {args.config} ({w.name}) run as a whole stream: {chunks} chunks, {L} layers, every chunk "
+                                                   f"timed after the windows have filled (chunk {fill}); plain calls, no graph",
+                                          l2="working set far exceeds L2; no flush", replicas="independent streams, no collective"),
+                              roofline=dict(bound="hbm", kernel="(whole step)", achieved=None, peak=None, unit=None, frac=None, traffic=None),
+                              cpu_baseline=None, e2e=None, gpu_launches=None, clocks=clocks,
+                              drift=dict(chunks_timed=len(lat), median_ms=float(np.median(lat)), first_5pct_ms=first, last_5pct_ms=last,
+                                         ratio_last_to_first=last / first, slope_ms_per_1000_chunks=slope,
+                                         max_ms=float(lat.max()), p99_ms=float(np.percentile(lat, 99)),
+                                         kept_tokens=int(len(meta["gids"])), max_position=int(meta["pos"].max()),
+                                         shift_total=int(meta["shift_total"])))))
+
+
 def dataclasses_replace(obj, **kw):
     import dataclasses
     return dataclasses.replace(obj, **kw)
@@ -819,9 +888,11 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="replay nothing: plain calls in the timed region")
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (smaller case for profiling)")
-    ap.add_argument("--workload", default="step", choices=["step", "overlap", "sweep", "qkv"],
+    ap.add_argument("--workload", default="step", choices=["step", "overlap", "sweep", "qkv", "drift"],
                     help="step: the per-chunk KV-cache step (default); overlap: the whole window re-prefilled every second; "
-                         "sweep: the step's latency over the paper's sink / window ablation values")
+                         "sweep: the step's latency over the paper's sink / window ablation values; qkv: the projection steps; "
+                         "drift: the config's whole stream, every chunk timed")
+    ap.add_argument("--chunks", type=int, default=0, help="drift: stream length in chunks (default: the config's)")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -873,6 +944,11 @@ def main():
         torch.cuda.synchronize()
 
     peaks = load_peaks()
+    if args.workload == "drift":
+        bench_drift(args, sg.workloads()[args.config], base, peaks, rank, world, local)
+        if world > 1:
+            dist.destroy_process_group()
+        return
     if args.workload == "qkv":
         bench_qkv(args, sg.workloads()[args.config], base, peaks, rank, world, local)
         if world > 1:
