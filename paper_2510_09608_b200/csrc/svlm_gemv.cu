@@ -8,6 +8,7 @@
 
 #include "svlm_dev.h"
 #include "svlm_launch.h"
+#include "svlm_ptx.cuh"
 
 namespace {
 
@@ -22,25 +23,33 @@ __global__ void __launch_bounds__(GV_THREADS) gemv_kernel(const uint16_t* __rest
     extern __shared__ __align__(16) unsigned char smem_raw[];
     uint4* sx = reinterpret_cast<uint4*>(smem_raw);            // [NX][in_dim / 8] chunks of 8 bf16; rows >= n are zero
     const int chunks = in_dim / 8;
+    const int lane = threadIdx.x & 31;
+    const int warp = blockIdx.x * (GV_THREADS / 32) + (threadIdx.x >> 5), n_warps = gridDim.x * (GV_THREADS / 32);
+    uint4 w[GV_UNROLL];
+    auto load_w = [&](int row, int c0) {
+        const uint4* wrow = reinterpret_cast<const uint4*>(W + (size_t)row * in_dim);
+#pragma unroll
+        for (int u = 0; u < GV_UNROLL; ++u) {
+            const int c = c0 + 32 * u;
+            w[u] = c < chunks ? __ldg(wrow + c) : make_uint4(0, 0, 0, 0);
+        }
+    };
+    // The weights do not depend on anything earlier in the stream: the kernel is launched while its predecessor
+    // may still run and fetches the first row of every warp at once; the token vectors wait for the predecessor.
+    svlm_ptx::pdl_launch_dependents();
+    if (warp < out_dim) load_w(warp, lane);
+    svlm_ptx::pdl_wait();
     for (int i = threadIdx.x; i < NX * chunks; i += GV_THREADS) {
         const int t = i / chunks;
         sx[i] = t < n ? *reinterpret_cast<const uint4*>(X + (size_t)t * in_dim + (size_t)(i % chunks) * 8) : make_uint4(0, 0, 0, 0);
     }
     __syncthreads();
-    const int lane = threadIdx.x & 31;
-    const int warp = blockIdx.x * (GV_THREADS / 32) + (threadIdx.x >> 5), n_warps = gridDim.x * (GV_THREADS / 32);
     for (int row = warp; row < out_dim; row += n_warps) {
-        const uint4* wrow = reinterpret_cast<const uint4*>(W + (size_t)row * in_dim);
         float acc[NX];
 #pragma unroll
         for (int t = 0; t < NX; ++t) acc[t] = 0.f;
         for (int c0 = lane; c0 < chunks; c0 += 32 * GV_UNROLL) {
-            uint4 w[GV_UNROLL];
-#pragma unroll
-            for (int u = 0; u < GV_UNROLL; ++u) {
-                const int c = c0 + 32 * u;
-                w[u] = c < chunks ? __ldg(wrow + c) : make_uint4(0, 0, 0, 0);
-            }
+            if (row != warp || c0 != lane) load_w(row, c0);      // the first batch is already here
 #pragma unroll
             for (int u = 0; u < GV_UNROLL; ++u) {
                 const int c = c0 + 32 * u;
@@ -138,8 +147,18 @@ cudaError_t launch(const uint16_t* X, const uint16_t* W, uint16_t* Y, int n, int
     const int rows_per_block = GV_THREADS / 32;
     int blocks = (out_dim + rows_per_block - 1) / rows_per_block;
     if (blocks > 2 * 148) blocks = 2 * 148;         // two resident blocks per SM, each warp walks a few rows
-    gemv_kernel<NX><<<blocks, GV_THREADS, smem, st>>>(X, W, Y, n, in_dim, out_dim);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(blocks);
+    cfg.blockDim = dim3(GV_THREADS);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // weights are fetched under the predecessor's tail
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    e = cudaLaunchKernelEx(&cfg, gemv_kernel<NX>, X, W, Y, n, in_dim, out_dim);
+    return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 }  // namespace
