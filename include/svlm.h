@@ -123,7 +123,7 @@ int svlm_qkv_append(svlm_cache* c, int layer, const void* X, const void* W, int 
  * side of a decode step: [q | k | v] = svlm_out_proj(x, W_qkv) is laid out as svlm_decode_step's Q, K and V.
  * Enqueued on the cache's stream (the cache is otherwise untouched).  in_dim a multiple of 64, out_dim a
  * multiple of 128, pointers 16-byte aligned.  Errors: SVLM_ERR_ARG.
- * Wo holds weights: with n <= 4 the kernel starts reading it while the work enqueued just before it on the
+ * Wo holds weights: with n <= 16 the kernel starts reading it while the work enqueued just before it on the
  * stream may still be running (only A waits for that work), so Wo must be complete in device memory before
  * that work starts; a kernel enqueued directly before this call must not be the one that writes Wo.
  */

@@ -109,13 +109,25 @@ __global__ void __launch_bounds__(GV_THREADS) gemv_mma_kernel(const uint16_t* __
     const bool lo_live = g < n, hi_live = g + 8 < n;
     const int n_kb = in_dim / 32;
     float c[4] = {0.f, 0.f, 0.f, 0.f};
+    uint4 w[GM_KB_IN_FLIGHT];
+    auto load_w = [&](int kb0) {
+#pragma unroll
+        for (int u = 0; u < GM_KB_IN_FLIGHT; ++u) {
+            const int kb = kb0 + u * (GV_THREADS / 32);
+            w[u] = kb < n_kb ? __ldg(wp + 4 * kb) : make_uint4(0, 0, 0, 0);
+        }
+    };
+    // as in the FMA form: the first batch of weights is fetched before the wait for the predecessor
+    svlm_ptx::pdl_launch_dependents();
+    load_w(warp);
+    svlm_ptx::pdl_wait();
     for (int kb0 = warp; kb0 < n_kb; kb0 += (GV_THREADS / 32) * GM_KB_IN_FLIGHT) {
-        uint4 w[GM_KB_IN_FLIGHT], a[GM_KB_IN_FLIGHT], bq[GM_KB_IN_FLIGHT];
+        uint4 a[GM_KB_IN_FLIGHT], bq[GM_KB_IN_FLIGHT];
+        if (kb0 != warp) load_w(kb0);
 #pragma unroll
         for (int u = 0; u < GM_KB_IN_FLIGHT; ++u) {
             const int kb = kb0 + u * (GV_THREADS / 32);
             const bool live = kb < n_kb;
-            w[u] = live ? __ldg(wp + 4 * kb) : make_uint4(0, 0, 0, 0);
             a[u] = live && lo_live ? __ldg(xlo + 4 * kb) : make_uint4(0, 0, 0, 0);
             bq[u] = live && hi_live ? __ldg(xhi + 4 * kb) : make_uint4(0, 0, 0, 0);
         }
@@ -173,8 +185,17 @@ cudaError_t svlm_launch_gemv(const void* X, const void* W, void* Y, int n, int i
     if (n == 1) e = launch<1>(x, w, y, n, in_dim, out_dim, st);
     else if (n <= 4) e = launch<4>(x, w, y, n, in_dim, out_dim, st);
     else {
-        gemv_mma_kernel<<<(out_dim + 7) / 8, GV_THREADS, 0, st>>>(x, w, y, n, in_dim, out_dim);
-        e = cudaGetLastError();
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((out_dim + 7) / 8);
+        cfg.blockDim = dim3(GV_THREADS);
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        e = cudaLaunchKernelEx(&cfg, gemv_mma_kernel, x, w, y, n, in_dim, out_dim);
+        if (e == cudaSuccess) e = cudaGetLastError();
     }
     svlm_count_launch();
     return e;
