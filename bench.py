@@ -791,6 +791,7 @@ def bench_qkv(args, wl, base, peaks, rank, world, local):
         wbytes = n_out * hidden * 2
         small.append(dict(n=n, ms_per_layer=ms, gbs=wbytes / (ms * 1e-3) / 1e9, frac_hbm=wbytes / (ms * 1e-3) / 1e9 / peaks["hbm"]))
     cache.close()
+    chain = decode_layer_chain(args, wl, peaks, rank, hidden, W, g)
     if rank == 0:
         d = rows[-1]
         roof = dict(bound="tensor", kernel="qkv_append", achieved=d["tflops"], peak=peaks["bf16_burst"], unit="TFLOP/s", frac=d["frac"],
@@ -801,7 +802,71 @@ def bench_qkv(args, wl, base, peaks, rank, world, local):
                                                    f"{wl.q_heads}+{wl.kv_heads}+{wl.kv_heads} heads of {wl.head_dim}, {L} layers in turn",
                                           l2="weights of the layers in turn exceed L2; no flush", replicas="independent streams, no collective"),
                               roofline=roof, cpu_baseline=None, e2e=None, gpu_launches=None, clocks=None, points=rows,
-                              decode_projection=small)))
+                              decode_projection=small, decode_layer_chain=chain)))
+
+
+def decode_layer_chain(args, wl, peaks, rank, hidden, W, g):
+    """One generated token through the attention half of every layer, as a decoder would call it:
+    [q | k | v] = W_qkv x (svlm_out_proj), the fused append + attention (svlm_decode_step), y = W_o a (svlm_out_proj),
+    the next layer's x being this layer's y; over the config's steady-state cache, one CUDA graph per token (the
+    position advances inside it), CUDA events around the replay.  All three kernels are launched while their
+    predecessor may still run and fetch what does not depend on it (weights, retained keys and values) first."""
+    import torch
+    from paper_2510_09608_b200 import binding
+    L = W.shape[0]
+    w = dataclasses_replace(wl, layers=L)
+    stream = sg.Stream(w, rank)
+    cache = binding.Cache(L, w.kv_heads, w.head_dim, w.n_sink, w.vision_window, w.text_window, w.capacity)
+    cache.set_rope(w.rope_mode, w.rope_base, w.sections)
+    fill_to_steady_state(cache, w, stream)
+    cache.evict()
+    qd = w.q_heads * w.head_dim
+    kd = w.kv_heads * w.head_dim
+    Wo = (torch.randn(L, hidden, qd, generator=g, device="cuda") / qd ** 0.5).to(torch.bfloat16)
+    x0 = torch.randn(1, hidden, generator=g, device="cuda").to(torch.bfloat16)
+    xs = [x0] + [torch.empty(1, hidden, dtype=torch.bfloat16, device="cuda") for _ in range(L)]
+    qkv = torch.empty(1, qd + 2 * kd, dtype=torch.bfloat16, device="cuda")
+    att = torch.empty(1, w.q_heads, w.head_dim, dtype=torch.bfloat16, device="cuda")
+    _, types, pos = stream.next_decode_token()
+    ty = torch.from_numpy(types).cuda()
+    pos_d = torch.from_numpy(np.ascontiguousarray(pos)).cuda()
+
+    def token():
+        for l in range(L):
+            cache.out_proj(xs[l], W[l], qkv)
+            cache.decode_step(l, qkv[:, qd:qd + kd].view(1, w.kv_heads, w.head_dim), qkv[:, qd + kd:].view(1, w.kv_heads, w.head_dim),
+                              ty, pos_d, qkv[:, :qd].view(1, w.q_heads, w.head_dim), att)
+            cache.out_proj(att.view(1, qd), Wo[l], xs[l + 1])
+        pos_d.add_(1)
+
+    token()                                  # plain once: one-time kernel attributes outside any capture
+    torch.cuda.synchronize()
+    cur = torch.cuda.current_stream()
+    gr = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(gr):
+        cache.set_stream(torch.cuda.current_stream())
+        token()
+    cache.set_stream(cur)
+    ts = []
+    n_tok = max(args.steps, 8)
+    for it in range(args.warmup + n_tok):
+        a, b2 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        gr.replay()
+        b2.record()
+        torch.cuda.synchronize()
+        if it >= args.warmup:
+            ts.append(a.elapsed_time(b2))
+    assert cache.status() == binding.OK
+    q = cache.query()
+    cache.close()
+    ms = statistics.median(ts)
+    # bytes a token must read per layer: both weight matrices and the retained keys and values, once
+    per_layer = (qd + 2 * kd) * hidden * 2 + hidden * qd * 2 + w.retained * 2 * kd * 2
+    return dict(ms_per_token=ms, us_per_layer=ms * 1e3 / L, tokens_per_s=1e3 / ms, layers=L,
+                bytes_per_layer=per_layer, gbs=per_layer * L / (ms * 1e-3) / 1e9,
+                frac_hbm=per_layer * L / (ms * 1e-3) / 1e9 / peaks["hbm"], kept_tokens=int(len(q["gids"])),
+                note="q/k/v projection + fused append and attention + output projection per layer, graph replay per token")
 
 
 def bench_drift(args, wl, base, peaks, rank, world, local):

@@ -25,7 +25,7 @@ def _run(*args):
     (["--config", "4", "--steps", "16", "--warmup", "3"], []),
     (["--config", "5", "--layers", "2", "--steps", "2", "--warmup", "3"], ["kernels"]),
     (["--workload", "overlap", "--layers", "2", "--steps", "3", "--warmup", "3"], ["kernels"]),
-    (["--workload", "qkv", "--layers", "2", "--steps", "2", "--warmup", "3"], ["points", "decode_projection"]),
+    (["--workload", "qkv", "--layers", "2", "--steps", "2", "--warmup", "3"], ["points", "decode_projection", "decode_layer_chain"]),
     (["--workload", "sweep", "--layers", "1"], ["sweep"]),
     (["--workload", "drift", "--layers", "2", "--chunks", "80"], ["drift"]),
 ])
