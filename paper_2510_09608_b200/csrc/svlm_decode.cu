@@ -129,9 +129,11 @@ decode_kernel(SvlmAttendBatch b, int layer0, int n_layers, const uint16_t* __res
     }
     // The metadata was written by an earlier kernel in the stream.  When the launcher vouches that
     // the kernel directly before this one did not write it (early_loads), it is read at once;
-    // otherwise after the grid-dependency wait.
-    pdl_launch_dependents();
+    // otherwise after the grid-dependency wait.  A kernel that has to wait does so BEFORE it lets its
+    // successor start: a successor with early loads then only ever runs behind a completed metadata
+    // kernel (whatever that kernel's own trigger), not merely behind one that has been launched.
     if (!early_loads) pdl_wait();
+    pdl_launch_dependents();
     const int n_tiles = min(__ldcg(&vw.ctrl->n_tiles), DEC_MAX_TILES);
     for (int i = threadIdx.x; i < n_tiles; i += DEC_THREADS) {
         const int4 tl = __ldcg(reinterpret_cast<const int4*>(vw.tiles + i));   // page, lo, hi, pad
