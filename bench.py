@@ -1203,7 +1203,7 @@ def main():
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        info = oracle_sample(wl)
+        info = oracle_sample(wl, layers=3)
         cpu = dict(value=frames_per_step / info["step_seconds"], unit="frames/s", cores=info["cores"], kind="oracle",
                    sample=info["sample"], est_ms_per_step=info["step_seconds"] * 1e3,
                    measured_seconds=info["measured_seconds"])
