@@ -147,7 +147,9 @@ int svlm_cache_evict(svlm_cache* c);
  * q_pos minus the total shift and sees every stored token whose ordinal does not exceed its own
  * (retained history fully, the new chunk causally).  Query head h reads KV head
  * h / (q_heads / kv_heads).  Scores are scaled by 1/sqrt(head_dim); a row that sees nothing yields
- * zeros.  n_q == 1 takes the split-KV decode path, n_q >= 2 the chunk-prefill path.
+ * zeros.  n_q == 1 takes the split-KV decode path, n_q >= 2 the chunk-prefill path; shapes neither of
+ * them is built for (more than 8 query heads per KV head at n_q == 1; a cache of more than 512 pages of 128
+ * slots, i.e. a capacity beyond roughly 65,000 tokens) take a slower general kernel with the same result.
  * Errors: SVLM_ERR_ARG (q_heads not a multiple of kv_heads, n_q < 1, null pointers),
  * SVLM_ERR_ORDER (n_q exceeds the tokens appended so far).
  */
@@ -165,7 +167,8 @@ int svlm_attend(svlm_cache* c, int layer, const void* Q, const int32_t* q_pos, i
  *               still needed: it is the query's position).
  * layer -1 takes all layers of the token in ONE launch, for callers that hold every layer's inputs at once (an
  * attention-only stack, a benchmark): K, V are [layers][kv_heads][head_dim], Q and out [layers][q_heads][head_dim].
- * At most 8 query heads per KV head.  Consecutive calls for different layers of the same token
+ * At most 8 query heads per KV head and at most 512 cache pages (a capacity up to roughly 65,000 tokens;
+ * beyond that SVLM_ERR_ARG: use svlm_cache_append + svlm_attend).  Consecutive calls for different layers of the same token
  * overlap on the GPU (the next layer's cache pages are fetched while the previous layer finishes);
  * K, V, Q and everything else produced by earlier work in the stream are read only after that work
  * has completed.
@@ -246,6 +249,7 @@ int svlm_decode_step_host(svlm_cache* c, int layer, const void* K_host, const vo
  *   - kv_heads x (number of KV splits: about one CTA per SM over the KV heads) x (16*head_dim + 64)
  *     bytes plus one counter per (layer, kv_head) must fit in it, otherwise SVLM_ERR_TOO_LARGE is
  *     returned and nothing runs (28 layers x 4 KV heads x head_dim 128 needs about 0.31 MB);
+ *   - the cache has at most 512 pages (capacity up to roughly 65,000 tokens), otherwise SVLM_ERR_TOO_LARGE;
  *   - all calls on one GPU share the array and it keeps the previous call's contents; the call
  *     clears what has to start at zero, on the cache's stream, before its kernel.  Calls whose
  *     kernels can overlap on the GPU (different streams, different caches) race on it: order them;

@@ -13,7 +13,7 @@ import numpy as np
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.environ.get("SVLM_LIBRARY") or os.path.join(_HERE, "libsvlm.so")   # SVLM_LIBRARY: a library built elsewhere
+LIB_PATH = os.path.join(_HERE, "libsvlm.so")
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2510_09608_b200.build`; "
@@ -23,6 +23,7 @@ _lib = C.CDLL(LIB_PATH)
 TEXT, VISION = 0, 1
 ROPE_1D, ROPE_MROPE = 0, 1
 OK, ERR_ARG, ERR_CAPACITY, ERR_ORDER, ERR_CUDA, ERR_TIMEOUT, ERR_NOMEM, ERR_TOO_LARGE = 0, -1, -2, -3, -4, -5, -6, -7
+NOALLOC_SCRATCH_BYTES = 512 << 10   # SVLM_NOALLOC_SCRATCH_BYTES of include/svlm.h
 
 _vp, _i, _i64p = C.c_void_p, C.c_int, C.POINTER(C.c_int64)
 _lib.svlm_cache_create.argtypes = [C.POINTER(_vp), _i, _i, _i, _i, _i, _i, _i]

@@ -546,6 +546,8 @@ size_t svlm_decode_ws_floats(int layers, int kv_heads, int head_dim, int splits)
     return (((size_t)layers * kv_heads + 3) & ~(size_t)3) + (size_t)layers * kv_heads * splits * pf;
 }
 
+bool svlm_decode_supported(int n_pages) { return n_pages <= DEC_MAX_TILES; }
+
 int svlm_decode_splits(int n_pages, int kv_heads, int problems) {
     // One problem (a single stream's layer): one CTA per SM, since the combine reads every split's
     // partial once and more splits than needed to fill the machine only lengthen the tail.  Several

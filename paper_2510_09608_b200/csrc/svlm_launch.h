@@ -45,6 +45,8 @@ void svlm_launch_attend_simple(const SvlmAttendBatch& b, int layer0, int n_layer
 // split-KV decode, n_q = 1 (svlm_decode.cu)
 size_t svlm_decode_ws_floats(int layers_in_launch, int kv_heads, int head_dim, int splits);
 int svlm_decode_splits(int n_pages, int kv_heads, int problems);
+// The kernel keeps the list of active pages in shared memory: caches with more pages take the general kernel.
+bool svlm_decode_supported(int n_pages);
 // Knew/Vnew non-null: fused decode step, the latest appended token's key and value ([caches*layers][kv_heads][d],
 // un-rotated) are written to the cache by this launch.  early_loads != 0: the caller vouches that no kernel
 // enqueued since the one before the previous launch on this stream wrote this cache's metadata or the pages of the

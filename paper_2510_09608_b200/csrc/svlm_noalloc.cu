@@ -60,6 +60,7 @@ extern "C" int svlm_attend_decode_noalloc(svlm_cache* c, int layer, const void* 
     const int group = q_heads / d.kv_heads;
     if (group > 8) return SVLM_ERR_ARG;                 // the split-KV kernel packs at most 8 query heads per KV head
     if (c->appended < 1) return SVLM_ERR_ORDER;
+    if (!svlm_decode_supported(d.n_pages)) return SVLM_ERR_TOO_LARGE;   // more pages than the kernel's page list holds
 
     const int splits = svlm_decode_splits(d.n_pages, d.kv_heads, 1);
     // counters for every (layer, kv head) of the cache, then one layer's partials
@@ -74,6 +75,9 @@ extern "C" int svlm_attend_decode_noalloc(svlm_cache* c, int layer, const void* 
     int rc = SVLM_OK;
     float* scratch = nullptr;
     rc = scratch_for_device(c->device, &scratch);
+    // What this call enqueues is not "a decode step of another layer" in the sense the regular entry points use to
+    // let their next launch read early: forget the record.
+    c->last_decode_layer = -1;
     if (rc == SVLM_OK) {
         // counters first in the scratch: they must be zero when the kernel starts
         const size_t counter_bytes = (size_t)d.layers * d.kv_heads * sizeof(unsigned);

@@ -219,7 +219,7 @@ int attend_common(svlm_cache* const* caches, int n_caches, int layer, const void
     } else {
         for (int i = 0; i < n_caches; ++i) caches[i]->last_decode_layer = -1;
     }
-    if (n_q == 1 && group <= 8) {
+    if (n_q == 1 && group <= 8 && svlm_decode_supported(c0->dev.n_pages)) {
         // split-KV decode; every cache's scratch was sized for this launch shape at creation
         const int splits = svlm_decode_splits(c0->dev.n_pages, c0->dev.kv_heads, n_caches * n_layers);
         SVLM_CUDA(svlm_launch_decode(b, layer0, n_layers, Q, q_pos, q_heads, out, splits, Knew, Vnew, early, c0->stream));
@@ -422,6 +422,8 @@ int svlm_out_proj(svlm_cache* c, const void* A, const void* Wo, int in_dim, int 
     if (!c || !A || !Wo || !Y || n < 1 || in_dim < 64 || in_dim % 64 || out_dim < 128 || out_dim % 128) return SVLM_ERR_ARG;
     if (((uintptr_t)A | (uintptr_t)Wo | (uintptr_t)Y) & 15) return SVLM_ERR_ARG;
     DeviceGuard guard(c->device);
+    // The cache's record of its latest decode launch stays as it is: this call neither reads nor writes the
+    // cache, so a decode step that follows may still fetch its pages early.
     if (svlm_gemv_supported(n, in_dim)) {      // a few tokens (decode): reading Wo once is all the work
         SVLM_CUDA(svlm_launch_gemv(A, Wo, Y, n, in_dim, out_dim, c->stream));
         return SVLM_OK;
@@ -472,6 +474,7 @@ int svlm_decode_step(svlm_cache* c, int layer, const void* K, const void* V, con
                      const int32_t* pos, const void* Q, int q_heads, void* out) {
     if (!c || !K || !V || !pos || !Q || !out || layer < -1 || layer >= c->dev.layers || q_heads < 1) return SVLM_ERR_ARG;
     if (q_heads % c->dev.kv_heads || q_heads / c->dev.kv_heads > 8) return SVLM_ERR_ARG;
+    if (!svlm_decode_supported(c->dev.n_pages)) return SVLM_ERR_ARG;   // more pages than the fused kernel's page list holds
     DeviceGuard guard(c->device);
     if (layer <= 0) {
         if (!token_type) return SVLM_ERR_ARG;
@@ -495,6 +498,7 @@ int svlm_decode_step_batched(svlm_cache* const* caches, int n_caches, int layer,
     svlm_cache* c0 = caches[0];
     if (!K || !V || !pos || !Q || !out || layer < 0 || layer >= c0->dev.layers || q_heads < 1) return SVLM_ERR_ARG;
     if (q_heads % c0->dev.kv_heads || q_heads / c0->dev.kv_heads > 8) return SVLM_ERR_ARG;
+    if (!svlm_decode_supported(c0->dev.n_pages)) return SVLM_ERR_ARG;
     DeviceGuard guard(c0->device);
     if (layer == 0) {
         if (!token_type) return SVLM_ERR_ARG;

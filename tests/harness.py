@@ -32,6 +32,50 @@ def dev_to_f64(t: torch.Tensor) -> np.ndarray:
     return t.float().cpu().numpy().astype(np.float64)
 
 
+class RotationCounter:
+    """Counts, per stored token, how often an eviction has moved its position, i.e. how many times
+    the library re-rotated (and re-rounded to bf16) its stored key after the first rotation.  Read
+    off the checker's metadata only: positions before and after each of its evictions."""
+
+    def __init__(self):
+        self.gids = np.zeros(0, np.int64)
+        self.count = np.zeros(0, np.int64)
+
+    def evict(self, ref):
+        before = ref.query()
+        ref.evict()
+        after = ref.query()
+        at = np.searchsorted(before["gids"], after["gids"])
+        assert np.array_equal(before["gids"][at], after["gids"])
+        moved = np.any(before["pos"][at] != after["pos"], axis=1)
+        old = np.zeros(len(after["gids"]), np.int64)
+        known = np.searchsorted(self.gids, after["gids"])
+        known = np.minimum(known, max(len(self.gids) - 1, 0))
+        if len(self.gids):
+            hit = self.gids[known] == after["gids"]
+            old[hit] = self.count[known[hit]]
+        self.gids, self.count = after["gids"], old + moved
+
+    def of(self, gids):
+        """Re-rotation counts of the given stored tokens (0 for tokens appended since the last eviction)."""
+        out = np.zeros(len(gids), np.int64)
+        if len(self.gids):
+            at = np.minimum(np.searchsorted(self.gids, gids), len(self.gids) - 1)
+            hit = self.gids[at] == gids
+            out[hit] = self.count[at[hit]]
+        return out
+
+
+def key_rounding_bound(want_k, roundings):
+    """Element-wise bound on |stored key - exact key|.  Every rotation ends in one rounding to bf16
+    (unit roundoff 2^-8), which moves a pair (x_i, x_{i+d/2}) by at most 2^-8 of the pair's norm, and
+    later rotations preserve that distance; `roundings` is the per-token number of roundings."""
+    half = want_k.shape[-1] // 2
+    pn = np.sqrt(want_k[..., :half] ** 2 + want_k[..., half:] ** 2)
+    pn = np.concatenate([pn, pn], axis=-1)
+    return np.asarray(roundings, np.float64)[:, None, None] * 2.0 ** -8 * 1.05 * pn + 1e-6
+
+
 class SideBySide:
     def __init__(self, wl: sg.Workload, stream: int = 0, layers=None, capacity=None, sink_any=False, contiguous=True):
         self.wl = wl
@@ -45,7 +89,7 @@ class SideBySide:
         self.ref = oracle.Oracle(self.layers, wl.kv_heads, wl.head_dim, wl.n_sink, wl.vision_window, wl.text_window,
                                  rope_mode=wl.rope_mode, rope_base=wl.rope_base, sections=wl.sections,
                                  sink_any_type=sink_any, contiguous=contiguous)
-        self.n_evicts = 0
+        self.rot = RotationCounter()
         self.last = None     # (gids, types, pos) of the latest append
 
     # -- steps ---------------------------------------------------------------------------------
@@ -109,8 +153,7 @@ class SideBySide:
 
     def evict(self):
         self.cache.evict()
-        self.ref.evict()
-        self.n_evicts += 1
+        self.rot.evict(self.ref)
 
     # -- checks --------------------------------------------------------------------------------
     def check_metadata(self):
@@ -128,18 +171,15 @@ class SideBySide:
         self.ref.set_kv(layer, gids, self.stream.k(layer, gids), self.stream.v(layer, gids))
 
     def check_kv(self, layer):
-        """Stored keys (rotated at the current positions) within the re-rotation bound; values exact."""
+        """Stored keys (rotated at the current positions) within each token's own re-rotation bound; values exact."""
         self._give_values_to_ref(layer)
         n = self.ref.count()
         Kb, Vb = self.cache.read_kv(layer, n)
         want_k, want_v = self.ref.rotated_k(layer), self.ref.values(layer)
         assert np.array_equal(sg.bf16_bits_to_f64(Vb), want_v), "values must be bit-exact"
         got_k = sg.bf16_bits_to_f64(Kb)
-        half = self.wl.head_dim // 2
-        pair_norm = np.sqrt(want_k[..., :half] ** 2 + want_k[..., half:] ** 2)
-        pair_norm = np.concatenate([pair_norm, pair_norm], axis=-1)
-        # every (re-)rotation rounds to bf16 once: |err| <= 2^-8 * pair norm per rounding
-        bound = (self.n_evicts + 1) * 2.0 ** -8 * 1.05 * pair_norm + 1e-6
+        # the first rotation plus this token's own re-rotations, one bf16 rounding each
+        bound = key_rounding_bound(want_k, 1 + self.rot.of(self.ref.query()["gids"]))
         err = np.abs(got_k - want_k)
         assert np.all(err <= bound), f"key error {err.max()} exceeds the rounding bound"
         return (float(err.max()), float(err.mean())) if err.size else (0.0, 0.0)

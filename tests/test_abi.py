@@ -22,3 +22,12 @@ def test_status_strings():
     assert binding.strerror(0) == "ok"
     for code in range(-6, 0):
         assert binding.strerror(code) != "unknown status"
+
+
+def test_binding_constants_match_the_header():
+    from paper_2510_09608_b200 import binding
+    header = open(os.path.join(ROOT, "include", "svlm.h")).read()
+    m = re.search(r"#define\s+SVLM_NOALLOC_SCRATCH_BYTES\s+\((\d+)u\s*<<\s*(\d+)\)", header)
+    assert m and binding.NOALLOC_SCRATCH_BYTES == int(m.group(1)) << int(m.group(2))
+    for name, value in re.findall(r"SVLM_(ERR_[A-Z_]+|OK)\s*=\s*(-?\d+)", header):
+        assert getattr(binding, name) == int(value), name

@@ -212,8 +212,7 @@ def test_batched_decode_steps_and_batched_evict(rope_1d):
         if step % 4 == 3:
             binding.evict_batched(caches)
             for s in sides:
-                s.ref.evict()
-                s.n_evicts += 1
+                s.rot.evict(s.ref)
                 s.check_metadata()
     for s in sides:
         s.check_metadata()
@@ -367,3 +366,88 @@ def test_errors_and_capacity():
                  torch.zeros(100, 1, 64, dtype=torch.bfloat16, device="cuda"),
                  torch.zeros(100, dtype=torch.uint8, device="cuda"), torch.arange(100, dtype=torch.int32, device="cuda"))
     assert e.value.status == binding.ERR_CAPACITY
+
+
+@pytest.mark.parametrize("contiguous", [True, False])
+def test_mrope_vision_window_that_cuts_a_block(contiguous):
+    """A vision window that is not a whole number of blocks: each chunk is one 2x8x8 block of 128 tokens and
+    the window holds 200, so the oldest retained block is always partly evicted.  The rule is applied
+    literally: a kept token moves left by the cursor advances of the evicted tokens before it, whatever
+    block they belong to, so a partly evicted block keeps its internal offsets."""
+    from harness import SideBySide, assert_close
+    wl = dataclasses.replace(_wl(2), layers=2, n_sink=24, vision_window=200, text_window=50,
+                             frames=2, grid_h=8, grid_w=8, text_max=24, decode_steps=2)
+    s = SideBySide(wl, contiguous=contiguous)
+    for chunk in range(10):
+        s.append_chunk(per_layer_calls=(chunk % 2 == 0))
+        s.evict()
+        n = s.check_metadata()
+        if chunk >= 2:
+            q = s.ref.query()
+            assert int((q["types"] == 1).sum()) == 200 and n == len(q["gids"])
+        s.check_kv(chunk % 2)
+        assert_close(s.attend(chunk % 2))
+        for _ in range(wl.decode_steps):
+            for st in s.decode_step_fused():
+                assert_close(st)
+    s.check_kv(0)
+    s.check_kv(1)
+
+
+@pytest.mark.parametrize("d,hq,hkv", [(128, 28, 2), (64, 12, 1)])
+def test_wide_gqa_group_decode_takes_the_general_kernel(d, hq, hkv):
+    """More than 8 query heads per KV head at n_q = 1 is outside the split-KV decode kernel: svlm_attend then runs
+    the general row-at-a-time kernel, and the fused decode step refuses the shape."""
+    from harness import SideBySide, assert_close, bits_to_dev
+    from paper_2510_09608_b200 import binding
+    base = _wl(2) if d == 128 else _wl(1)
+    wl = dataclasses.replace(base, layers=2, q_heads=hq, kv_heads=hkv, n_sink=10, vision_window=3 * 64, text_window=40,
+                             frames=1, grid_h=8, grid_w=8, text_max=12, decode_steps=2, head_dim=d)
+    s = SideBySide(wl)
+    for chunk in range(6):
+        s.append_chunk()
+        s.evict()
+        s.check_metadata()
+        assert_close(s.attend(chunk % 2))                   # chunk prefill: the tensor-core kernel takes any group
+        for _ in range(wl.decode_steps):
+            s.append_decode_token()
+            assert_close(s.attend(chunk % 2))               # n_q = 1, group 14 / 12: general kernel
+            assert_close(s.attend(0, all_layers=True))
+    gids, types, pos = s.stream.next_decode_token()
+    with pytest.raises(binding.SvlmError) as e:
+        s.cache.decode_step(0, bits_to_dev(s.stream.k(0, gids)), bits_to_dev(s.stream.v(0, gids)),
+                            torch.from_numpy(types).cuda(), torch.from_numpy(np.ascontiguousarray(pos)).cuda(),
+                            bits_to_dev(s.stream.q(0, gids)))
+    assert e.value.status == binding.ERR_ARG
+    s.check_metadata()                                       # the refused call changed nothing
+
+
+def test_cache_with_more_pages_than_the_fast_kernels_list():
+    """A capacity beyond 512 pages (no-eviction or full-attention style use): one-token attention over all of
+    it must not stop at the 512th page.  svlm_attend takes the general kernel for both shapes; the fused decode
+    step and the no-allocation entry point refuse."""
+    from harness import SideBySide, assert_close, bits_to_dev
+    from paper_2510_09608_b200 import binding
+    n_chunk = 4 * 32 * 32                                    # 4096 vision tokens per chunk
+    wl = dataclasses.replace(_wl(1), layers=1, q_heads=2, kv_heads=1, n_sink=0, vision_window=1 << 20, text_window=1 << 20,
+                             frames=4, grid_h=32, grid_w=32, text_max=8, decode_steps=1)
+    s = SideBySide(wl, capacity=66 * 1024 + 512)
+    for chunk in range(16):                                  # 65.5k vision tokens + text: 513+ pages in use
+        s.append_chunk()
+    s.evict()
+    n = s.check_metadata()
+    assert n > 512 * 128
+    rows = np.array([0, n_chunk // 2, len(s.last[0]) - 1])
+    assert_close(s.attend(0, rows=rows))                     # n_q >= 2 over more than 512 pages
+    s.append_decode_token()
+    assert_close(s.attend(0))                                # n_q = 1 over more than 512 pages
+    gids, types, pos = s.stream.next_decode_token()
+    args = (bits_to_dev(s.stream.k(0, gids)), bits_to_dev(s.stream.v(0, gids)), torch.from_numpy(types).cuda(),
+            torch.from_numpy(np.ascontiguousarray(pos)).cuda(), bits_to_dev(s.stream.q(0, gids)))
+    with pytest.raises(binding.SvlmError) as e:
+        s.cache.decode_step(0, *args)
+    assert e.value.status == binding.ERR_ARG
+    with pytest.raises(binding.SvlmError) as e:
+        s.cache.attend_decode_noalloc(0, args[4], args[3])
+    assert e.value.status == binding.ERR_TOO_LARGE
+    s.check_metadata()

@@ -180,3 +180,78 @@ def test_tiny_stream_equals_brute_force_over_kept_set(mode):
             vis = kept[None, :] <= (n_before + np.arange(n))[:, None]
             want = brute.attention(qrot, krot, vall[kept, g], vis)
             assert np.allclose(got[:, h], want, atol=1e-12), (step, h)
+
+
+@pytest.mark.parametrize("mode", [ROPE_1D, ROPE_MROPE])
+def test_late_values_and_row_subsets_equal_brute_force(mode):
+    """The two entry points the long-stream GPU tests lean on: values handed over after the fact by
+    stream ordinal (`set_kv`, shuffled, with ordinals that are no longer stored mixed in) and the
+    `rows` subset of `attend`.  Pinned against dense numpy attention over the closed-form kept set,
+    against the same stream fed with values at append time, and against the full-row result."""
+    rng = np.random.default_rng(23 + mode)
+    hq, hkv, d, S, Vw, Tw, L = 6, 2, 8, 2, 8, 3, 2
+    sections = (2, 1, 1)
+    kw = dict(rope_mode=mode, rope_base=100.0, sections=sections)
+    early = Oracle(L, hkv, d, S, Vw, Tw, **kw)     # K/V supplied with the append
+    late = Oracle(L, hkv, d, S, Vw, Tw, **kw)      # metadata only; K/V by set_kv before attending
+    items, types_hist, Ks, Vs = [], [], [], []
+    for step in range(10):
+        new = [("V", 1, 2, 2)] + [("T",)] * int(rng.integers(0, 4))
+        n_before = len(types_hist)
+        items += new
+        tnew = [VISION] * 4 + [TEXT] * (len(new) - 1)
+        types_hist += tnew
+        n = len(tnew)
+        if mode == ROPE_MROPE:
+            native = brute.assign_positions(items)
+            pos = native[n_before:].astype(np.int32)
+        else:
+            native = np.repeat(np.arange(len(types_hist))[:, None], 3, 1)
+            pos = native[n_before:, 0].astype(np.int32)
+        K, V = _bits(rng.standard_normal((L, n, hkv, d))), _bits(rng.standard_normal((L, n, hkv, d)))
+        Q = _bits(rng.standard_normal((n, hq, d)))
+        Ks.append(K); Vs.append(V)
+        early.append(K, V, np.array(tnew, np.uint8), pos)
+        late.append(None, None, np.array(tnew, np.uint8), pos)
+        early.evict(); late.evict()
+        kall, vall = np.concatenate(Ks, axis=1), np.concatenate(Vs, axis=1)    # [L, history, hkv, d]
+        mask = brute.kept_mask(np.array(types_hist), S, Vw, Tw)
+        kept = np.flatnonzero(mask)
+        assert np.array_equal(late.query()["gids"], kept)
+        if step < 2:
+            continue
+        layer = step % L
+        # before any value arrives (or with one stored token left out) attention must refuse
+        if step in (2, 3):
+            with pytest.raises(RuntimeError):
+                late.attend(layer, Q, pos)
+            hole = kept[kept != kept[len(kept) // 2]]
+            late.set_kv(layer, hole, kall[layer, hole], vall[layer, hole])
+            with pytest.raises(RuntimeError):
+                late.attend(layer, Q, pos)
+        # every ordinal of the history in shuffled order: the evicted ones must be skipped silently
+        order = rng.permutation(len(types_hist))
+        late.set_kv(layer, order, kall[layer, order], vall[layer, order])
+        assert np.array_equal(late.query()["gids"], kept), "set_kv must not change what is stored"
+        full_early = early.attend(layer, Q, pos)
+        full_late = late.attend(layer, Q, pos)
+        assert np.allclose(full_late, full_early, atol=1e-12)
+        rows = rng.permutation(n)[: max(1, n // 2)]
+        sub = late.attend(layer, Q, pos, rows=rows)
+        assert sub.shape == (len(rows), hq, d)
+        assert np.allclose(sub, full_late[rows], atol=1e-12)
+        assert np.allclose(early.attend(layer, Q, pos, rows=rows[::-1]), full_early[rows[::-1]], atol=1e-12)
+        # dense numpy over the closed-form kept set, for the chosen rows only
+        adv = np.diff(np.maximum.accumulate(np.concatenate([[0], native.max(1) + 1])))
+        freed = np.where(mask, 0, adv)
+        cpos = native - (np.cumsum(freed) - freed)[:, None]
+        total_freed = int(freed.sum())
+        sec = sections if mode == ROPE_MROPE else None
+        kf, vf, qf = sg.bf16_bits_to_f64(kall[layer]), sg.bf16_bits_to_f64(vall[layer]), sg.bf16_bits_to_f64(Q)
+        for h in range(hq):
+            g = h // (hq // hkv)
+            krot = np.stack([brute.rope(kf[j, g], cpos[j], 100.0, sec) for j in kept])
+            qrot = np.stack([brute.rope(qf[r, h], native[n_before + r] - total_freed, 100.0, sec) for r in rows])
+            vis = kept[None, :] <= (n_before + rows)[:, None]
+            want = brute.attention(qrot, krot, vf[kept, g], vis)
+            assert np.allclose(sub[:, h], want, atol=1e-12), (step, h)
