@@ -938,6 +938,92 @@ def bench_drift(args, wl, base, peaks, rank, world, local):
                                          shift_total=int(meta["shift_total"])))))
 
 
+TRACE_STATIONS = {0: "kernel entry", 1: "page list in shared memory", 2: "first round's copies issued",
+                  3: "previous kernel complete (dependency wait returns)", 4: "rotated query in shared memory",
+                  5: "warp 1 has its keys", 14: "warp 1: scores and softmax done", 6: "warp 1 through with its units",
+                  7: "all consumer warps through", 8: "CTA's record written", 9: "arrival counted",
+                  10: "combining CTA: records staged", 11: "combining CTA: output written", 13: "CTA leaves"}
+
+
+def bench_decode_trace(args, wl, base, peaks, rank, world, local):
+    """In-kernel time stamps of the layer-sequential decode chain: the instrumented build of the library
+    (paper_2510_09608_b200.build.build_trace) runs generated tokens through svlm_decode_step, one launch per layer,
+    replayed from a CUDA graph as in the step benchmark, and every CTA's thread 0 records %globaltimer at the
+    stations of the chain.  Prints, per station, the median and the latest CTA's time relative to the moment the
+    dependency wait returns, averaged over the traced launches that could read ahead (every layer but a token's first)."""
+    import ctypes
+    import torch
+    from paper_2510_09608_b200 import binding
+    lib = binding._lib
+    if not hasattr(lib, "svlm_debug_decode_trace_start"):
+        raise SystemExit("decode-trace needs the instrumented library: python -m paper_2510_09608_b200.build --trace")
+    L = wl.layers
+    stream = sg.Stream(wl, rank)
+    cache = binding.Cache(L, wl.kv_heads, wl.head_dim, wl.n_sink, wl.vision_window, wl.text_window, wl.capacity)
+    cache.set_rope(wl.rope_mode, wl.rope_base, wl.sections)
+    fill_to_steady_state(cache, wl, stream)
+    cache.evict()
+    n_tok = max(2, 56 // L)
+    w1 = dataclasses_replace(wl, decode_steps=n_tok)
+    inp = StepInputs(w1, stream, *next_step_schedule(stream, w1))
+    run_step(cache, w1, inp)                        # plain once: kernel attributes, warm caches
+    torch.cuda.synchronize()
+    inp = StepInputs(w1, stream, *next_step_schedule(stream, w1))
+
+    def tokens():
+        for d in inp.dec:
+            for l in range(L):
+                cache.decode_step(l, d["K"][l], d["V"][l], d["types"] if l == 0 else None, d["pos"], d["Q"][l], d["out"][l])
+
+    lib.svlm_debug_decode_trace_start.restype = None
+    lib.svlm_debug_decode_trace_start()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        cache.set_stream(torch.cuda.current_stream())
+        tokens()
+    cache.set_stream(torch.cuda.current_stream())
+    a, b2 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    g.replay()
+    b2.record()
+    torch.cuda.synchronize()
+    assert cache.status() == binding.OK
+    buf = np.zeros((64, 160, 16), np.uint64)
+    assert lib.svlm_debug_decode_trace_read(buf.ctypes.data_as(ctypes.c_void_p)) == 0
+    t = buf.astype(np.int64)
+    rows, periods = [], []
+    prev_w = None
+    for i in range(min(64, n_tok * L)):
+        n = int((t[i, :, 0] > 0).sum())
+        if n == 0:
+            break
+        x = t[i, :n]
+        w = float(np.median(x[:, 3]))
+        early = bool(np.median(x[:, 0]) < w - 2000)      # entered well before the wait returned: it could read ahead
+        if prev_w is not None and early:
+            periods.append((w - prev_w) / 1e3)
+        prev_w = w
+        if early:
+            rows.append({k: ((float(np.median(x[:, k][x[:, k] > 0])) - w) / 1e3, (float(x[:, k].max()) - w) / 1e3)
+                         for k in TRACE_STATIONS if (x[:, k] > 0).any()})
+    table = []
+    for k, name in TRACE_STATIONS.items():
+        vals = [r[k] for r in rows if k in r]
+        if vals:
+            table.append(dict(station=name, median_us=round(float(np.mean([v[0] for v in vals])), 2),
+                              latest_cta_us=round(float(np.mean([v[1] for v in vals])), 2)))
+    table.sort(key=lambda r: r["latest_cta_us"])
+    if rank == 0:
+        print(json.dumps(dict(base, metric="decode layer-step period (instrumented build)", unit="us", higher_is_better=False,
+                              value=float(np.mean(periods)) if periods else None,
+                              ms_per_step=a.elapsed_time(b2) / n_tok,
+                              config=dict(workload=f"config {args.config} shape, {L} layers: {n_tok} generated tokens, one svlm_decode_step "
+                                                   f"launch per layer, graph replay; timer resolution about 0.26 us; the stamps themselves add "
+                                                   f"a little to the chain"),
+                              roofline=None, cpu_baseline=None, e2e=None, gpu_launches=n_tok * (L + 1), clocks=None,
+                              launches_traced=len(rows), trace=table)))
+
+
 def dataclasses_replace(obj, **kw):
     import dataclasses
     return dataclasses.replace(obj, **kw)
@@ -955,10 +1041,11 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="replay nothing: plain calls in the timed region")
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (smaller case for profiling)")
-    ap.add_argument("--workload", default="step", choices=["step", "overlap", "sweep", "qkv", "drift"],
+    ap.add_argument("--workload", default="step", choices=["step", "overlap", "sweep", "qkv", "drift", "decode-trace"],
                     help="step: the per-chunk KV-cache step (default); overlap: the whole window re-prefilled every second; "
                          "sweep: the step's latency over the paper's sink / window ablation values; qkv: the projection steps; "
-                         "drift: the config's whole stream, every chunk timed")
+                         "drift: the config's whole stream, every chunk timed; decode-trace: in-kernel time stamps of the "
+                         "decode chain (needs the instrumented build of the library)")
     ap.add_argument("--chunks", type=int, default=0, help="drift: stream length in chunks (default: the config's)")
     args = ap.parse_args()
 
@@ -1003,6 +1090,10 @@ def main():
 
     import torch
     import torch.distributed as dist
+    if args.workload == "decode-trace":
+        import paper_2510_09608_b200 as pkg
+        from paper_2510_09608_b200 import build as _build
+        pkg.LIB_OVERRIDE = _build.build_trace()       # the instrumented build, before the binding loads a library
     from paper_2510_09608_b200 import binding
 
     torch.cuda.set_device(local)
@@ -1015,6 +1106,11 @@ def main():
         torch.cuda.synchronize()
 
     peaks = load_peaks()
+    if args.workload == "decode-trace":
+        bench_decode_trace(args, wl, base, peaks, rank, world, local)
+        if world > 1:
+            dist.destroy_process_group()
+        return
     if args.workload == "drift":
         bench_drift(args, sg.workloads()[args.config], base, peaks, rank, world, local)
         if world > 1:

@@ -279,6 +279,17 @@ int svlm_cache_read_kv(svlm_cache* c, int layer, void* K_host, void* V_host);
 /* Sticky device-side status (SVLM_OK if nothing went wrong).  Synchronises the cache's stream. */
 int svlm_cache_status(svlm_cache* c);
 
+/*
+ * Debugging aid: the number of polls a bounded device-side wait of this cache's kernels makes before it
+ * gives up (every wait inside the kernels is bounded; one that runs out makes its thread block record
+ * SVLM_ERR_TIMEOUT in the sticky status, wait for its copies in flight, release what it holds and return).
+ * The default, 2^20 polls, is seconds; 0 makes every wait give up at once, which is how the tests walk
+ * the give-up paths without anything actually hanging.  The results of calls that timed out are
+ * undefined; the cache's metadata and stored K/V are not touched by the attention kernels and stay valid,
+ * but the sticky status stays set for the life of the cache.  Synchronises the cache's stream.
+ */
+int svlm_debug_set_wait_limit(svlm_cache* c, unsigned polls);
+
 /* Number of kernels this library has launched in this process (all caches). */
 int64_t svlm_launch_count(void);
 

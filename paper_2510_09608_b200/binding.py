@@ -13,7 +13,9 @@ import numpy as np
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libsvlm.so")
+from . import LIB_OVERRIDE as _override
+
+LIB_PATH = _override or os.path.join(_HERE, "libsvlm.so")
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2510_09608_b200.build`; "
@@ -49,6 +51,7 @@ _lib.svlm_attend_decode_noalloc.argtypes = [_vp, _i, _vp, _vp, _i, _vp]
 _lib.svlm_cache_query.argtypes = [_vp, _i64p, _vp, _vp, _vp, _i64p]
 _lib.svlm_cache_read_kv.argtypes = [_vp, _i, _vp, _vp]
 _lib.svlm_cache_status.argtypes = [_vp]
+_lib.svlm_debug_set_wait_limit.argtypes = [_vp, C.c_uint]
 _lib.svlm_launch_count.restype = C.c_int64
 _lib.svlm_strerror.restype = C.c_char_p
 _lib.svlm_strerror.argtypes = [_i]
@@ -225,6 +228,9 @@ class Cache:
 
     def status(self) -> int:
         return int(_lib.svlm_cache_status(self._h))
+
+    def debug_set_wait_limit(self, polls: int):
+        _check(_lib.svlm_debug_set_wait_limit(self._h, int(polls)), "svlm_debug_set_wait_limit")
 
 
 def attend_batched(caches, layer, Q, q_pos, out=None):

@@ -48,5 +48,27 @@ def build(force: bool = False, verbose: bool = False) -> str:
     return LIB
 
 
+def build_trace() -> str:
+    """A second library, libsvlm_trace.so, whose decode kernel stamps %globaltimer at the stations of its chain
+    (compile-time switch SVLM_DECODE_TRACE in csrc/svlm_decode.cu).  Only the benchmark's decode-trace workload
+    loads it; the product library is untouched."""
+    build()
+    out = os.path.join(HERE, "libsvlm_trace.so")
+    src = os.path.join(CSRC, "svlm_decode.cu")
+    obj = os.path.join(BUILD, "svlm_decode_trace.o")
+    newest = max([os.path.getmtime(src)] + [os.path.getmtime(h) for h in _headers()])
+    if not os.path.exists(obj) or os.path.getmtime(obj) < newest:
+        res = subprocess.run(["nvcc", *NVCC_FLAGS, "-DSVLM_DECODE_TRACE", "-c", src, "-o", obj], capture_output=True, text=True)
+        if res.returncode:
+            sys.stderr.write(res.stdout + res.stderr)
+            raise RuntimeError("nvcc failed on the trace build of " + src)
+    others = [os.path.join(BUILD, os.path.basename(f)[:-3] + ".o") for f in _sources() if not f.endswith("svlm_decode.cu")]
+    if not os.path.exists(out) or any(os.path.getmtime(o) > os.path.getmtime(out) for o in [obj] + others):
+        subprocess.check_call(["nvcc", "-shared", "-o", out, obj, *others, "-lcudart"])
+    return out
+
+
 if __name__ == "__main__":
     print(build(force="--force" in sys.argv, verbose=True))
+    if "--trace" in sys.argv:
+        print(build_trace())

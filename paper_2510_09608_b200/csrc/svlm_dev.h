@@ -33,7 +33,7 @@ struct SvlmCtrl {            // one per cache, device memory; only meta kernels 
     int status;              // sticky svlm_status
     int append_n;            // tokens staged by the latest metadata append (0 if it was dropped)
     int evict_moved;         // 1 if the latest evict shifted any retained token
-    int pad;
+    unsigned wait_limit;     // polls a bounded device-side wait makes before it gives up (set at creation)
 };
 
 struct SvlmTile {            // one active page as the attention kernels see it
@@ -67,7 +67,7 @@ struct SvlmCacheDev {        // passed by value to kernels
     uint16_t* V;             // same shape, as appended
     float* ws;               // split-KV partials
     void* tmaps;             // TMA descriptors (device memory, 4 x 128 bytes): K, V slabs with a 128-row box
-                             // (chunk prefill), then K, V with a 32-row box (decode)
+                             // (chunk prefill), then K, V with a 32-row box (batched decode)
     float* rope_tab;         // [3][256][head_dim/2] (cos, sin) pairs, see svlm_rope.cuh
     double theta[SVLM_MAX_HALF];   // base^(-2i/head_dim)
 };

@@ -173,6 +173,7 @@ prefill_kernel(SvlmAttendBatch b, int layer0, int n_layers, const uint16_t* __re
     const int n_tiles = min(vw.ctrl->n_tiles, PF_MAX_TILES);
     const long long gid_q0 = vw.ctrl->n_total - n_q;
     const long long shift = vw.ctrl->shift_total;
+    const unsigned wait_limit = vw.ctrl->wait_limit;
 
     // ---- set-up: barriers, TMEM, page list ------------------------------------------------------
     if (threadIdx.x == 0) {
@@ -218,7 +219,7 @@ prefill_kernel(SvlmAttendBatch b, int layer0, int n_layers, const uint16_t* __re
             const int y = (int)(head_row0 + (size_t)(t & 0x3FFF) * SVLM_PAGE);
             const int kv = pr_n & 1;      // even items are K pages, odd items V pages of the same page
             const int st = pr_n % PF_RING;
-            pr_ok = mbar_wait(&sh.empty[st], ((pr_n / PF_RING) & 1) ^ 1, abort_flag);   // first pass: already free
+            pr_ok = mbar_wait(&sh.empty[st], ((pr_n / PF_RING) & 1) ^ 1, abort_flag, wait_limit);   // first pass: already free
             if (!pr_ok) break;
             mbar_expect_tx(&sh.full[st], TILE_BYTES);
 #pragma unroll
@@ -372,7 +373,7 @@ prefill_kernel(SvlmAttendBatch b, int layer0, int n_layers, const uint16_t* __re
             // every wait gives the same answer in all lanes, so the warp stays converged
             auto wait_bar = [&](void* bar, unsigned parity) {   // one lane polls, all lanes get the answer
                 int r = 1;
-                if (lane == 0) r = mbar_wait(bar, parity, abort_flag);
+                if (lane == 0) r = mbar_wait(bar, parity, abort_flag, wait_limit);
                 return __shfl_sync(0xffffffffu, r, 0) != 0;
             };
             auto wait_item = [&](int n) { return wait_bar(&sh.full[n % PF_RING], (n / PF_RING) & 1); };
@@ -472,7 +473,7 @@ prefill_kernel(SvlmAttendBatch b, int layer0, int n_layers, const uint16_t* __re
                 vlo = tl.lo;
                 vlen = a - tl.lo;
             }
-            ok = mbar_wait(&sh.s_full[g], it & 1, abort_flag);
+            ok = mbar_wait(&sh.s_full[g], it & 1, abort_flag, wait_limit);
             if (!ok) break;
             tc_fence_after();
             float rowsum, corr, m_new;
@@ -485,7 +486,7 @@ prefill_kernel(SvlmAttendBatch b, int layer0, int n_layers, const uint16_t* __re
             mbar_arrive(&sh.p_full[g]);
             ++it;
         }
-        if (ok) ok = mbar_wait(&sh.all_done, 0, abort_flag);
+        if (ok) ok = mbar_wait(&sh.all_done, 0, abort_flag, wait_limit);
         tc_fence_after();
 
         // ---- hand-over between the two CTAs of the cluster, then the output ------------------------

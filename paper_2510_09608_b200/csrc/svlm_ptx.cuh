@@ -6,7 +6,8 @@
 
 namespace svlm_ptx {
 
-constexpr unsigned WAIT_LIMIT = 1u << 20;   // polls before a wait gives up (seconds at worst)
+constexpr unsigned WAIT_LIMIT = 1u << 20;   // default number of polls before a wait gives up (seconds at worst);
+                                            // the limit in force is a field of the cache's control block
 
 __device__ __forceinline__ unsigned smem_u32(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
 
@@ -26,9 +27,10 @@ __device__ __forceinline__ bool mbar_test(void* bar, unsigned parity) {
                  : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
     return ok != 0;
 }
-// Bounded wait: false when the limit ran out or another thread of the CTA already gave up.
-__device__ __forceinline__ bool mbar_wait(void* bar, unsigned parity, volatile int* abort_flag) {
-    for (unsigned it = 0; it < WAIT_LIMIT; ++it) {
+// Bounded wait: false when `limit` polls ran out (a limit of 0 gives up at once, whatever the barrier's
+// state) or another thread of the CTA already gave up.
+__device__ __forceinline__ bool mbar_wait(void* bar, unsigned parity, volatile int* abort_flag, unsigned limit) {
+    for (unsigned it = 0; it < limit; ++it) {
         if (mbar_test(bar, parity)) return true;
         if ((it & 63) == 63) {
             if (*abort_flag) return false;

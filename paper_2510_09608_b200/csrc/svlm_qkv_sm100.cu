@@ -71,6 +71,7 @@ qkv_append_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
     const int m0 = blockIdx.y * 128;             // first token of the tile
     const int n_kb = hidden / QK_BK;
     volatile int* abort_flag = &sh.abort_flag;
+    const unsigned wait_limit = cd.ctrl->wait_limit;   // written at creation only, never by a kernel
 
     if (smem_u32(smem_raw) & 1023) {             // swizzled tiles need a 1024-byte aligned base; same in every CTA
         if (threadIdx.x == 0) atomicCAS(&cd.ctrl->status, 0, -4);   // SVLM_ERR_CUDA
@@ -96,7 +97,7 @@ qkv_append_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
         if (lane == 0) {
             for (int kb = 0; kb < n_kb; ++kb) {
                 const int st = kb % QK_STAGES;
-                if (!mbar_wait(&sh.empty[st], ((kb / QK_STAGES) & 1) ^ 1, abort_flag)) break;   // first pass: already free
+                if (!mbar_wait(&sh.empty[st], ((kb / QK_STAGES) & 1) ^ 1, abort_flag, wait_limit)) break;   // first pass: already free
                 unsigned char* dst = ring + st * QK_STAGE;
                 mbar_expect_tx(&sh.full[st], QK_STAGE);
                 tma_load_2d(dst, &tmX, kb * QK_BK, m0, &sh.full[st]);                 // rows past the end read as zeros
@@ -111,7 +112,7 @@ qkv_append_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
             bool ok = true;
             for (int kb = 0; kb < n_kb && ok; ++kb) {
                 const int st = kb % QK_STAGES;
-                ok = mbar_wait(&sh.full[st], (kb / QK_STAGES) & 1, abort_flag);
+                ok = mbar_wait(&sh.full[st], (kb / QK_STAGES) & 1, abort_flag, wait_limit);
                 if (!ok) break;
                 tc_fence_after();
                 const unsigned long long da = smem_desc(smem_u32(ring + st * QK_STAGE), 16, 1024);
@@ -153,7 +154,7 @@ qkv_append_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant
                 }
             }
         }
-        const bool ok = mbar_wait(&sh.acc_full, 0, abort_flag);
+        const bool ok = mbar_wait(&sh.acc_full, 0, abort_flag, wait_limit);
         tc_fence_after();
 #pragma unroll 1
         for (int hh = 0; hh < 2 && ok; ++hh) {

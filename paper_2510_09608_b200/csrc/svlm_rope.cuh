@@ -14,6 +14,14 @@ __device__ __forceinline__ float2 svlm_cmul(float2 a, float2 b) {
     return make_float2(a.x * b.x - a.y * b.y, a.x * b.y + a.y * b.x);
 }
 
+// Positions beyond the table's range: fp64 sincos, kept out of line (its argument reduction is a lot of code
+// that the callers' instruction stream should not have to carry).
+static __device__ __noinline__ float2 svlm_rope_cs_far(double angle) {
+    double s, co;
+    sincos(angle, &s, &co);
+    return make_float2((float)co, (float)s);
+}
+
 // tab: [3][256][half] float2.  Returns (cos, sin) of c * theta where theta belongs to `pair`.
 __device__ __forceinline__ float2 svlm_rope_cs(const float2* __restrict__ tab, int half, int pair, long long c,
                                                double theta) {
@@ -27,9 +35,7 @@ __device__ __forceinline__ float2 svlm_rope_cs(const float2* __restrict__ tab, i
             if (u >> 16) r = svlm_cmul(r, __ldg(tab + (size_t)(512 + (u >> 16)) * half + pair));
         }
     } else {
-        double s, co;
-        sincos((double)a * theta, &s, &co);
-        r = make_float2((float)co, (float)s);
+        r = svlm_rope_cs_far((double)a * theta);
     }
     if (c < 0) r.y = -r.y;
     return r;

@@ -8,6 +8,7 @@
 #include <algorithm>
 #include <atomic>
 #include <cmath>
+#include <cstddef>
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
@@ -306,6 +307,7 @@ int svlm_cache_create(svlm_cache** out, int layers, int kv_heads, int head_dim, 
         SvlmCtrl ctrl;
         std::memset(&ctrl, 0, sizeof ctrl);
         ctrl.free_top = (int)stack.size();
+        ctrl.wait_limit = 1u << 20;   // polls; seconds at worst
         std::vector<long long> minus1(d.n_slots, -1);
         if (cudaMemcpy(d.free_stack, stack.data(), stack.size() * sizeof(int), cudaMemcpyHostToDevice) != cudaSuccess ||
             cudaMemcpy(d.ctrl, &ctrl, sizeof ctrl, cudaMemcpyHostToDevice) != cudaSuccess ||
@@ -743,6 +745,16 @@ int svlm_cache_status(svlm_cache* c) {
     SvlmCtrl ctrl;
     SVLM_CUDA(cudaMemcpy(&ctrl, c->dev.ctrl, sizeof ctrl, cudaMemcpyDeviceToHost));
     return ctrl.status;
+}
+
+int svlm_debug_set_wait_limit(svlm_cache* c, unsigned polls) {
+    if (!c) return SVLM_ERR_ARG;
+    DeviceGuard guard(c->device);
+    c->wait_limit_host = polls;   // the copy reads this field when the stream reaches it
+    SVLM_CUDA(cudaMemcpyAsync(reinterpret_cast<char*>(c->dev.ctrl) + offsetof(SvlmCtrl, wait_limit), &c->wait_limit_host,
+                              sizeof(unsigned), cudaMemcpyHostToDevice, c->stream));
+    SVLM_CUDA(cudaStreamSynchronize(c->stream));
+    return SVLM_OK;
 }
 
 int64_t svlm_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
