@@ -226,6 +226,52 @@ def run_step_multi(caches, wl, inps, dec, timers=None, pre=None):
         timed("decode_token", lambda: decode_token(d))
 
 
+def run_step_host_layered(cache, wl, inp):
+    """The step of run_step through the host-buffer entry points, layer by layer as a decoder calls them: every
+    call copies its own inputs up from pinned host memory, and the attention calls bring their output down before
+    they return."""
+    h = inp.h
+    cache.append_host(0, h["K"][0], h["V"][0], h["types"], h["pos"])
+    cache.evict()
+    cache.attend_host(0, h["Q"][0], h["pos"], h["out"][0])
+    for l in range(1, wl.layers):
+        cache.append_host(l, h["K"][l], h["V"][l], None, None)
+        cache.attend_host(l, h["Q"][l], h["pos"], h["out"][l])
+    for d in inp.hdec:
+        for l in range(wl.layers):
+            cache.decode_step_host(l, d["K"][l], d["V"][l], d["types"] if l == 0 else None, d["pos"], d["Q"][l], d["out"][l])
+
+
+def time_decode_tokens(cache, wl, inp, replays=3):
+    """Milliseconds per generated token for the decode part of a step as the step benchmark runs it (one fused
+    svlm_decode_step launch per layer, replayed from a CUDA graph): the token launches of `inp` are captured once and
+    replayed; an eviction between replays keeps the cache at its steady-state size.  Median of the replays after the
+    first (which carries the graph's upload)."""
+    import torch
+
+    def tokens():
+        for d in inp.dec:
+            for l in range(wl.layers):
+                cache.decode_step(l, d["K"][l], d["V"][l], d["types"] if l == 0 else None, d["pos"], d["Q"][l], d["out"][l])
+
+    g = torch.cuda.CUDAGraph()
+    cur = torch.cuda.current_stream()
+    with torch.cuda.graph(g):
+        cache.set_stream(torch.cuda.current_stream())
+        tokens()
+    cache.set_stream(cur)
+    ts = []
+    for _ in range(replays + 1):
+        cache.evict()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        g.replay()
+        b.record()
+        torch.cuda.synchronize()
+        ts.append(a.elapsed_time(b) / max(len(inp.dec), 1))
+    return statistics.median(ts[1:])
+
+
 def run_step_host(cache, wl, inp):
     """The same step through the host-buffer entry points (all layers per call): copies included."""
     cache.append_host(-1, inp.h["K"], inp.h["V"], inp.h["types"], inp.h["pos"])
@@ -260,15 +306,27 @@ def fill_to_steady_state(cache, wl, stream):
     return chunks
 
 
-# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the attention and eviction kernels from the
-# ncu captures summarised under profiles/ (*_kernel_config3_8layers.txt; one layer per attention launch, so the
-# per-launch traffic is that of the full 28-layer run; the evict launch covers 8 layers there and is scaled by the
-# layer count).  Set an entry to None when its kernel changes until the counters are taken again.
-NCU_DRAM_BYTES = {
-    "decode": 19.07e6,                 # one layer's K and V once (algorithmic: 18.9 MB)
-    "prefill": 22.94e6,                # one layer's K and V once plus Q and the output (the rest is served by L2)
-    "evict_per_layer": (71.4e6 + 15.4e6) / 8,   # reads all re-rotated keys; most of the write-back is still in L2 at kernel end
-}
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the attention and eviction kernels come from
+# the ncu captures summarised under profiles/: profiles/ncu_dram_traffic.txt lists, per kernel, the bytes per launch on
+# the config-3 shape, the source file the kernel lives in and that file's SHA-256 at the time of the capture.  A kernel
+# whose source has changed since reports no traffic (null) until its counters are taken again.
+def ncu_dram_traffic():
+    import hashlib
+    out = {}
+    path = os.path.join(ROOT, "profiles", "ncu_dram_traffic.txt")
+    if not os.path.exists(path):
+        return out
+    for line in open(path):
+        f = line.split()
+        if len(f) < 4 or line.startswith("#"):
+            continue
+        name, nbytes, src, digest = f[0], float(f[1]), f[2], f[3]
+        try:
+            now = hashlib.sha256(open(os.path.join(ROOT, src), "rb").read()).hexdigest()
+        except OSError:
+            now = None
+        out[name] = nbytes if now == digest else None
+    return out
 
 
 def max_over_ranks(value: float, world: int, device="cuda") -> float:
@@ -671,12 +729,17 @@ def bench_sweep(args, wl, base, peaks, rank, world, local):
     points += [("sink", v, wl.text_window, wl.vision_window) for v in (0, 64, 256, 1024)]
     points += [("text_window", wl.n_sink, v, wl.vision_window) for v in (0, 64, 256, 1024)]
     points += [("vision_window", wl.n_sink, wl.text_window, sec * per_s) for sec in (0, 1, 4, 8, 32)]
+    # the policy switches at the deployed sizes (the paper's Table 4 arms as latency): native positions instead of
+    # contiguous ones (eviction then only releases storage: no key is re-rotated), and sinks of any token type
+    points += [("policy:native_rope", wl.n_sink, wl.text_window, wl.vision_window),
+               ("policy:sink_any_type", wl.n_sink, wl.text_window, wl.vision_window)]
     rows = []
     for axis, S, Tw, Vw in points:
         w = dataclasses_replace(wl, layers=L, n_sink=S, text_window=Tw, vision_window=Vw)
         stream = sg.Stream(w, rank)
         cache = binding.Cache(L, w.kv_heads, w.head_dim, S, Vw, Tw, w.capacity)
         cache.set_rope(w.rope_mode, w.rope_base, w.sections)
+        cache.set_policy(sink_any_type=(axis == "policy:sink_any_type"), contiguous=(axis != "policy:native_rope"))
         fill_to_steady_state(cache, w, stream)
         cache.evict()
         timers = {}
@@ -698,10 +761,10 @@ def bench_sweep(args, wl, base, peaks, rank, world, local):
         nq = int(round(statistics.mean(n_q)))
         flops = prefill_flops(w, nq, lk) if lk >= nq else float("nan")   # the chunk itself is (partly) evicted: no closed form
         kv_bytes = kept * 2 * w.kv_heads * w.head_dim * 2
-        moved = max(kept - w.decode_steps - S, 0)
+        moved = max(kept - w.decode_steps - S, 0) if axis != "policy:native_rope" else 0
         ev_bytes = 2 * moved * w.kv_heads * w.head_dim * 2 * L
         step_ms = sum(tot.values())
-        rows.append(dict(axis=axis, n_sink=S, text_window=Tw, vision_window_s=Vw // per_s, kept_tokens=kept,
+        rows.append(dict(axis=axis, contiguous=(axis != "policy:native_rope"), sink_any_type=(axis == "policy:sink_any_type"), n_sink=S, text_window=Tw, vision_window_s=Vw // per_s, kept_tokens=kept,
                          step_ms=step_ms, evict_ms=avg["evict"], prefill_ms=avg["prefill"],
                          decode_layer_step_ms=avg["decode_token"] / L,
                          prefill_frac=(flops / (avg["prefill"] * 1e-3) / 1e12 / peaks["bf16_burst"]) if flops == flops else None,
@@ -945,6 +1008,92 @@ TRACE_STATIONS = {0: "kernel entry", 1: "page list in shared memory", 2: "first 
                   10: "combining CTA: records staged", 11: "combining CTA: output written", 13: "CTA leaves"}
 
 
+def bench_drift_multi(args, wl, base, peaks, rank, world, local):
+    """bench_drift for a workload of several streams in lock step (config 5: 8 streams, 7200 chunks = two hours of
+    8 frames/s video each): per chunk every stream appends its tokens, ONE batched eviction, per layer the appends and
+    ONE chunk-prefill launch for all streams, then the generated tokens with one batched decode launch per layer;
+    every chunk of all streams is timed by its own event pair.  Values are drawn once and reused; token types, counts
+    and positions follow each stream."""
+    import torch
+    from paper_2510_09608_b200 import binding
+    L = args.layers or wl.layers
+    w = dataclasses_replace(wl, layers=L)
+    S = w.streams
+    chunks = args.chunks or w.chunks
+    streams = [sg.Stream(w, rank * S + i) for i in range(S)]
+    caches, fill = [], 0
+    for st in streams:
+        c = binding.Cache(L, w.kv_heads, w.head_dim, w.n_sink, w.vision_window, w.text_window, w.capacity)
+        c.set_rope(w.rope_mode, w.rope_base, w.sections)
+        fill = fill_to_steady_state(c, w, st)
+        c.evict()
+        caches.append(c)
+    g = torch.Generator(device="cuda").manual_seed(w.seed)
+    nmax = w.max_chunk_tokens
+    rnd = lambda *shape: torch.randn(*shape, generator=g, device="cuda").to(torch.bfloat16)  # noqa: E731
+    K, V = rnd(L, nmax, w.kv_heads, w.head_dim), rnd(L, nmax, w.kv_heads, w.head_dim)
+    Q = rnd(L, S * nmax, w.q_heads, w.head_dim)
+    out = torch.empty_like(Q)
+    k1, v1, q1 = rnd(L, S, w.kv_heads, w.head_dim), rnd(L, S, w.kv_heads, w.head_dim), rnd(L, S, w.q_heads, w.head_dim)
+    o1 = torch.empty_like(q1)
+    text1 = torch.zeros(S, dtype=torch.uint8, device="cuda")
+    sampler = ClockSampler(local)
+    sampler.start()
+    evs = []
+    for i in range(chunks - fill):
+        sched = [st.next_chunk() for st in streams]
+        n_q = [len(sc[0]) for sc in sched]
+        tys = [torch.from_numpy(sc[1]).cuda() for sc in sched]
+        pss = [torch.from_numpy(np.ascontiguousarray(sc[2])).cuda() for sc in sched]
+        pos_all = torch.cat(pss).contiguous()
+        tot = sum(n_q)
+        dec = []
+        for _ in range(w.decode_steps):
+            toks = [st.next_decode_token() for st in streams]
+            dec.append(torch.from_numpy(np.ascontiguousarray(np.stack([t[2][0] for t in toks]))).cuda())
+        a, b2 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for c, n, ty, ps in zip(caches, n_q, tys, pss):
+            c.append(0, K[0, :n], V[0, :n], ty, ps)
+        binding.evict_batched(caches)
+        for l in range(L):
+            if l:
+                for c, n in zip(caches, n_q):
+                    c.append(l, K[l, :n], V[l, :n])
+            binding.attend_batched_varlen(caches, l, Q[l, :tot], pos_all, n_q, out[l, :tot])
+        for p1 in dec:
+            for l in range(L):
+                binding.decode_step_batched(caches, l, k1[l], v1[l], text1 if l == 0 else None, p1, q1[l], o1[l])
+        b2.record()
+        evs.append((a, b2))
+        if i % 32 == 31:
+            torch.cuda.synchronize()      # keep the host from running far ahead of the device
+    torch.cuda.synchronize()
+    clocks = sampler.finish()
+    for c in caches:
+        assert c.status() == binding.OK
+    metas = [c.query() for c in caches]
+    lat = np.array([a.elapsed_time(b2) for a, b2 in evs])
+    k5 = max(1, len(lat) // 20)
+    first, last = float(np.median(lat[:k5])), float(np.median(lat[-k5:]))
+    slope = float(np.polyfit(np.arange(len(lat)), lat, 1)[0]) * 1000.0
+    if rank == 0:
+        med = float(np.median(lat))
+        print(json.dumps(dict(base, value=w.frames * S / (med * 1e-3), ms_per_step=med, steps=len(lat),
+                              config=dict(workload=f"config {args.config} ({w.name}) run as whole streams: {S} streams in lock step, {chunks} chunks "
+                                                   f"each, {L} layers, every chunk (of all streams) timed after the windows have filled "
+                                                   f"(chunk {fill}); plain calls, no graph",
+                                          l2="working set far exceeds L2; no flush", replicas="independent streams, no collective"),
+                              roofline=dict(bound="hbm", kernel="(whole step)", achieved=None, peak=None, unit=None, frac=None, traffic=None),
+                              cpu_baseline=None, e2e=None, gpu_launches=None, clocks=clocks,
+                              drift=dict(chunks_timed=len(lat), median_ms=med, first_5pct_ms=first, last_5pct_ms=last,
+                                         ratio_last_to_first=last / first, slope_ms_per_1000_chunks=slope,
+                                         max_ms=float(lat.max()), p99_ms=float(np.percentile(lat, 99)),
+                                         kept_tokens=[int(len(m["gids"])) for m in metas],
+                                         max_position=int(max(m["pos"].max() for m in metas)),
+                                         shift_total=[int(m["shift_total"]) for m in metas]))))
+
+
 def bench_decode_trace(args, wl, base, peaks, rank, world, local):
     """In-kernel time stamps of the layer-sequential decode chain: the instrumented build of the library
     (paper_2510_09608_b200.build.build_trace) runs generated tokens through svlm_decode_step, one launch per layer,
@@ -1020,7 +1169,9 @@ def bench_decode_trace(args, wl, base, peaks, rank, world, local):
                               config=dict(workload=f"config {args.config} shape, {L} layers: {n_tok} generated tokens, one svlm_decode_step "
                                                    f"launch per layer, graph replay; timer resolution about 0.26 us; the stamps themselves add "
                                                    f"a little to the chain"),
-                              roofline=None, cpu_baseline=None, e2e=None, gpu_launches=n_tok * (L + 1), clocks=None,
+                              roofline=dict(bound="hbm", kernel="decode (instrumented)", achieved=None, peak=None, unit=None, frac=None,
+                                            traffic=None),
+                              cpu_baseline=None, e2e=None, gpu_launches=n_tok * (L + 1), clocks=None,
                               launches_traced=len(rows), trace=table)))
 
 
@@ -1112,7 +1263,8 @@ def main():
             dist.destroy_process_group()
         return
     if args.workload == "drift":
-        bench_drift(args, sg.workloads()[args.config], base, peaks, rank, world, local)
+        wd = sg.workloads()[args.config]
+        (bench_drift_multi if wd.streams > 1 else bench_drift)(args, wd, base, peaks, rank, world, local)
         if world > 1:
             dist.destroy_process_group()
         return
@@ -1228,15 +1380,21 @@ def main():
     torch.cuda.synchronize()
     prefill_ms = ea.elapsed_time(eb) / wl.layers
     flops_b = prefill_flops(wl, inp_b.n, lk)
+    # The decode launches as the step runs them: graph replay of one step's generated tokens (a separately timed
+    # plain call would carry the host's launch gaps).
+    decode_token_ms = time_decode_tokens(cache, wl, prof_inputs[-1]) if wl.decode_steps else float("nan")
     kernels = {
         "prefill": dict(bound="tensor", avg_ms=prefill_ms, per_step_ms=prefill_ms * wl.layers,
                         achieved=flops_b / (prefill_ms * 1e-3) / 1e12, unit="TFLOP/s", peak=peaks["bf16_burst"],
                         single_call_ms=avg["prefill"], note="avg_ms = the layers' launches back to back / layers"),
         # one launch per layer; the launches of one token overlap (programmatic dependent launch), so the
         # per-launch duration is the token's time over its L launches (the metadata launch is inside it)
-        "decode": dict(bound="hbm", avg_ms=avg["decode_token"] / wl.layers, per_step_ms=tot["decode_token"],
-                       achieved=kv_bytes_layer * wl.layers / (avg["decode_token"] * 1e-3) / 1e9, unit="GB/s",
-                       peak=peaks["hbm"], note="avg_ms = time of one token's decode over all layers / layers"),
+        "decode": dict(bound="hbm", avg_ms=decode_token_ms / wl.layers, per_step_ms=decode_token_ms * wl.decode_steps,
+                       achieved=kv_bytes_layer * wl.layers / (decode_token_ms * 1e-3) / 1e9, unit="GB/s",
+                       peak=peaks["hbm"], plain_call_ms=avg["decode_token"] / wl.layers,
+                       note="avg_ms = time of one token's decode over all layers / layers, graph replay of 16 tokens as in "
+                            "the step (one launch per layer, the metadata launch inside); plain_call_ms: the same by "
+                            "separately timed calls"),
         "evict": dict(bound="hbm", avg_ms=avg["evict"], per_step_ms=tot["evict"],
                       achieved=evict_bytes / (avg["evict"] * 1e-3) / 1e9, unit="GB/s", peak=peaks["hbm"]),
         "append": dict(avg_ms=avg["append"], per_step_ms=tot["append"]),
@@ -1247,9 +1405,10 @@ def main():
         kernels[k]["frac_of_nominal"] = kernels[k]["achieved"] / (2250.0 if kernels[k]["bound"] == "tensor" else 8000.0)
     dominant = max(("prefill", "decode", "evict"), key=lambda k: kernels[k]["per_step_ms"])
     kd = kernels[dominant]
-    traffic = NCU_DRAM_BYTES.get(dominant)
-    if dominant == "evict" and NCU_DRAM_BYTES.get("evict_per_layer") is not None:
-        traffic = NCU_DRAM_BYTES["evict_per_layer"] * wl.layers
+    ncu_bytes = ncu_dram_traffic()
+    traffic = ncu_bytes.get(dominant)
+    if dominant == "evict":
+        traffic = ncu_bytes["evict_per_layer"] * wl.layers if ncu_bytes.get("evict_per_layer") is not None else None
     if args.config not in (2, 3):
         traffic = None          # the counters were taken on the config-3 shape
     roofline = dict(bound="tensor" if dominant == "prefill" else "hbm", kernel=dominant, achieved=kd["achieved"],
@@ -1283,20 +1442,29 @@ def main():
 
     # ---- end to end through the host-buffer entry points -----------------------------------------
     e2e = None
+    e2e_all_layers = None
     if want_e2e:
         hin = [StepInputs(wl, stream, *next_step_schedule(stream, wl), host=True) for _ in range(3)]
         e2e_steps = min(args.steps, 5)
-        run_step_host(cache, wl, hin[0])
-        barrier()
-        t0 = time.perf_counter()
-        for i in range(e2e_steps):
-            run_step_host(cache, wl, hin[1 + i % 2])
-        torch.cuda.synchronize()
-        e2e_s = (time.perf_counter() - t0) / e2e_steps
-        e2e_s = max_over_ranks(e2e_s, world)
-        e2e = dict(value=whole_job_value(world, frames_per_step, e2e_s * 1e3), unit="frames/s", ms_per_step=e2e_s * 1e3,
+
+        def timed_host(fn):
+            fn(cache, wl, hin[0])
+            barrier()
+            t0 = time.perf_counter()
+            for i in range(e2e_steps):
+                fn(cache, wl, hin[1 + i % 2])
+            torch.cuda.synchronize()
+            return max_over_ranks((time.perf_counter() - t0) / e2e_steps, world)
+
+        lay_s = timed_host(run_step_host_layered)
+        all_s = timed_host(run_step_host)
+        e2e = dict(value=whole_job_value(world, frames_per_step, lay_s * 1e3), unit="frames/s", ms_per_step=lay_s * 1e3,
                    h2d_bytes_per_step=hin[1].h2d_bytes(), d2h_bytes_per_step=hin[1].d2h_bytes(),
-                   api="svlm_cache_append_host / svlm_attend_host / svlm_decode_step_host, all layers per call, pinned host buffers")
+                   api="svlm_cache_append_host / svlm_attend_host / svlm_decode_step_host, one call per layer as in `value` "
+                       "(each attention call returns with its output in host memory), pinned host buffers")
+        e2e_all_layers = dict(value=whole_job_value(world, frames_per_step, all_s * 1e3), unit="frames/s", ms_per_step=all_s * 1e3,
+                              api="the same entry points with all layers per call (layer = -1): the chunk prefill pipelines the "
+                                  "layers' copies, a generated token is one launch")
 
     elapsed_ms = max_over_ranks(elapsed_ms, world)
     ms_per_step = elapsed_ms / args.steps
@@ -1312,8 +1480,8 @@ def main():
         third = max(1, args.steps // 3)
         line = dict(base, value=whole_job_value(world, frames_per_step, ms_per_step), ms_per_step=ms_per_step, config=config,
                     roofline=roofline, cpu_baseline=cpu, e2e=e2e, gpu_launches=int(gpu_launches), clocks=clocks,
-                    kernels=kernels, decode_tok_s=wl.decode_steps / (tot["decode_token"] * 1e-3),
-                    decode_all_layers_one_launch=all_layers,
+                    kernels=kernels, decode_tok_s=1e3 / decode_token_ms,
+                    decode_all_layers_one_launch=all_layers, e2e_all_layers_per_call=e2e_all_layers,
                     step_ms=dict(min=min(step_ms), median=statistics.median(step_ms), max=max(step_ms),
                                  first_third=statistics.median(step_ms[:third]),
                                  last_third=statistics.median(step_ms[-third:])),
