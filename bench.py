@@ -308,7 +308,7 @@ def fill_to_steady_state(cache, wl, stream):
 
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the attention and eviction kernels come from
 # the ncu captures summarised under profiles/: profiles/ncu_dram_traffic.txt lists, per kernel, the bytes per launch on
-# the config-3 shape, the source file the kernel lives in and that file's SHA-256 at the time of the capture.  A kernel
+# the config-3 shape, the source files the kernel is built from and their SHA-256 at the time of the capture.  A kernel
 # whose source has changed since reports no traffic (null) until its counters are taken again.
 def ncu_dram_traffic():
     import hashlib
@@ -321,8 +321,8 @@ def ncu_dram_traffic():
         if len(f) < 4 or line.startswith("#"):
             continue
         name, nbytes, src, digest = f[0], float(f[1]), f[2], f[3]
-        try:
-            now = hashlib.sha256(open(os.path.join(ROOT, src), "rb").read()).hexdigest()
+        try:      # src: the kernel's files joined by '+', hashed one after another
+            now = hashlib.sha256(b"".join(open(os.path.join(ROOT, x), "rb").read() for x in src.split("+"))).hexdigest()
         except OSError:
             now = None
         out[name] = nbytes if now == digest else None
