@@ -451,3 +451,29 @@ def test_cache_with_more_pages_than_the_fast_kernels_list():
         s.cache.attend_decode_noalloc(0, args[4], args[3])
     assert e.value.status == binding.ERR_TOO_LARGE
     s.check_metadata()
+
+
+@pytest.mark.parametrize("d", [64, 128])
+def test_per_layer_decode_with_several_rounds_per_cta(d):
+    """A cache large enough, over few enough CTAs, that a CTA of the per-layer decode kernel holds more 16-key units
+    than its six warps take in one round (8 KV heads: 18 CTAs per head; more than 40 pages in use): the second round
+    reuses the warps' slots and carries the running maximum.  Plain and fused decode steps of every layer."""
+    from harness import SideBySide, assert_close
+    base = _wl(2) if d == 128 else _wl(1)
+    wl = dataclasses.replace(base, layers=2, q_heads=16, kv_heads=8, head_dim=d, n_sink=100, vision_window=6 * 1024, text_window=300,
+                             frames=4, grid_h=16, grid_w=16, text_max=24, decode_steps=2)
+    s = SideBySide(wl)
+    for chunk in range(8):
+        s.append_chunk()
+        s.evict()
+    n = s.check_metadata()
+    assert n > 48 * 128          # 8 units per page over 18 CTAs: more than the 18 units of one round
+    for step in range(3):
+        if step % 2:
+            for st in s.decode_step_fused():
+                assert_close(st)
+        else:
+            s.append_decode_token()
+            assert_close(s.attend(0))
+            assert_close(s.attend(1))
+    s.check_kv(1)

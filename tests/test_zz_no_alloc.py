@@ -93,3 +93,43 @@ def test_noalloc_limit_both_sides():
                 cache.attend_decode_noalloc(0, Q, qp)
             assert e.value.status == binding.ERR_TOO_LARGE
         cache.close()
+
+
+def test_noalloc_between_fused_decode_steps_changes_nothing():
+    """The no-allocation call enqueued between two layers' fused decode steps: the steps must give what they give
+    without it (the regular entry points start reading a layer's pages early only behind a decode of another layer of
+    the same cache, and the no-allocation call is not one of those)."""
+    from harness import bits_to_dev, dev_to_f64
+    from paper_2510_09608_b200 import binding, streamgen as sg
+
+    wl = dataclasses.replace(sg.workloads()[2], layers=3, n_sink=40, vision_window=5 * 128, text_window=70,
+                             frames=2, grid_h=8, grid_w=8, text_max=24)
+
+    def run(interleave):
+        stream = sg.Stream(wl, 0)
+        cache = binding.Cache(wl.layers, wl.kv_heads, wl.head_dim, wl.n_sink, wl.vision_window, wl.text_window, wl.capacity)
+        cache.set_rope(wl.rope_mode, wl.rope_base, wl.sections)
+        for _ in range(6):
+            gids, types, pos = stream.next_chunk()
+            K = np.stack([stream.k(l, gids) for l in range(wl.layers)])
+            V = np.stack([stream.v(l, gids) for l in range(wl.layers)])
+            cache.append(-1, bits_to_dev(K), bits_to_dev(V), torch.from_numpy(types).cuda(), torch.from_numpy(np.ascontiguousarray(pos)).cuda())
+            cache.evict()
+        outs = []
+        for _ in range(2):
+            gids, types, pos = stream.next_decode_token()
+            ty, ps = torch.from_numpy(types).cuda(), torch.from_numpy(np.ascontiguousarray(pos)).cuda()
+            for l in range(wl.layers):
+                outs.append(dev_to_f64(cache.decode_step(l, bits_to_dev(stream.k(l, gids)), bits_to_dev(stream.v(l, gids)),
+                                                         ty if l == 0 else None, ps, bits_to_dev(stream.q(l, gids)))))
+                if interleave:      # attention of the same token over another layer, through the fixed scratch array
+                    other = (l + 2) % wl.layers
+                    if other < l:   # only layers whose K/V of this token are already in the cache
+                        cache.attend_decode_noalloc(other, bits_to_dev(stream.q(other, gids)), ps)
+        assert cache.status() == binding.OK
+        cache.close()
+        return outs
+
+    plain, mixed = run(False), run(True)
+    for a, b in zip(plain, mixed):
+        assert np.array_equal(a, b)
