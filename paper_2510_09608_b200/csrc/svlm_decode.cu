@@ -86,6 +86,9 @@ constexpr int UPW = 3;                              // units per warp and round
 constexpr int GROUP = DEC_CWARPS * UPW;             // units per round
 constexpr int LAY_SLOTS = UPW + 1;                  // private slots per warp: the round's key units + one value unit
 constexpr int MERGE_PAD = 4;                        // floats of padding per head row of the merge buffer
+// The rotated query rows sit D + 8 elements apart in shared memory: the MMA fragment loads (lane = head * 4 + pair of
+// dims) then hit 32 different banks; with rows D apart the eight heads of a load collide on four banks.
+constexpr int QROW_PAD = 8;
 
 __device__ __forceinline__ void ldmatrix_x4(unsigned& r0, unsigned& r1, unsigned& r2, unsigned& r3, const void* p) {
     const unsigned s = (unsigned)__cvta_generic_to_shared(p);
@@ -332,7 +335,7 @@ decode_stream_kernel(SvlmAttendBatch b, int layer0, int n_layers, const uint16_t
     unsigned char* ring = reinterpret_cast<unsigned char*>(
         (reinterpret_cast<uintptr_t>(smem_raw) + sizeof(DecShared) + 1023) & ~(uintptr_t)1023);
     uint16_t* s_q = reinterpret_cast<uint16_t*>(ring + DEC_STAGES * STAGE_BYTES);   // [8][D] bf16
-    uint16_t* s_new = s_q + 8 * D;       // fused step: the new token's rotated key [D], then its value [D]
+    uint16_t* s_new = s_q + 8 * (D + QROW_PAD);       // fused step: the new token's rotated key [D], then its value [D]
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int g = lane >> 2, t = lane & 3;
@@ -478,8 +481,8 @@ decode_stream_kernel(SvlmAttendBatch b, int layer0, int n_layers, const uint16_t
                 if (h >= 8) continue;
                 const float x = h < G ? __bfloat162float(__ushort_as_bfloat16(qx[k])) : 0.f;
                 const float y = h < G ? __bfloat162float(__ushort_as_bfloat16(qy[k])) : 0.f;
-                s_q[h * D + pair] = __bfloat16_as_ushort(__float2bfloat16_rn(x * cs.x - y * cs.y));
-                s_q[h * D + pair + HALF] = __bfloat16_as_ushort(__float2bfloat16_rn(y * cs.x + x * cs.y));
+                s_q[h * (D + QROW_PAD) + pair] = __bfloat16_as_ushort(__float2bfloat16_rn(x * cs.x - y * cs.y));
+                s_q[h * (D + QROW_PAD) + pair + HALF] = __bfloat16_as_ushort(__float2bfloat16_rn(y * cs.x + x * cs.y));
             }
             if (prep_new) {
                 const float x = __bfloat162float(__ushort_as_bfloat16(kx)), y = __bfloat162float(__ushort_as_bfloat16(ky));
@@ -493,8 +496,8 @@ decode_stream_kernel(SvlmAttendBatch b, int layer0, int n_layers, const uint16_t
         unsigned qf[KSTEPS][2];   // B fragments of Q^T: (d = ks*16 + 2t.., head g)
 #pragma unroll
         for (int ks = 0; ks < KSTEPS; ++ks) {
-            qf[ks][0] = *reinterpret_cast<const unsigned*>(s_q + g * D + ks * 16 + 2 * t);
-            qf[ks][1] = *reinterpret_cast<const unsigned*>(s_q + g * D + ks * 16 + 2 * t + 8);
+            qf[ks][0] = *reinterpret_cast<const unsigned*>(s_q + g * (D + QROW_PAD) + ks * 16 + 2 * t);
+            qf[ks][1] = *reinterpret_cast<const unsigned*>(s_q + g * (D + QROW_PAD) + ks * 16 + 2 * t + 8);
         }
 
         const float scale = 1.4426950408889634f * rsqrtf((float)D);
@@ -638,7 +641,7 @@ decode_stream_kernel(SvlmAttendBatch b, int layer0, int n_layers, const uint16_t
 
 template <int D>
 constexpr size_t decode_stream_smem() {
-    return sizeof(DecShared) + 1024 + (size_t)DEC_STAGES * 2 * SUB * D * 2 + 8 * D * 2 + 2 * D * 2;
+    return sizeof(DecShared) + 1024 + (size_t)DEC_STAGES * 2 * SUB * D * 2 + 8 * (D + QROW_PAD) * 2 + 2 * D * 2;
 }
 static_assert(merge_bytes<128>() <= (size_t)DEC_STAGES * 2 * SUB * 128 * 2 && merge_bytes<64>() <= (size_t)DEC_STAGES * 2 * SUB * 64 * 2,
               "the merge slabs live in the ring");
@@ -674,7 +677,7 @@ decode_layer_kernel(SvlmAttendBatch b, int layer, const uint16_t* __restrict__ Q
     unsigned char* ring = reinterpret_cast<unsigned char*>(
         (reinterpret_cast<uintptr_t>(smem_raw) + sizeof(LayShared) + 127) & ~(uintptr_t)127);
     uint16_t* s_q = reinterpret_cast<uint16_t*>(ring + RING_BYTES);   // [8][D] bf16
-    uint16_t* s_new = s_q + 8 * D;       // fused step: the new token's rotated key [D], then its value [D]
+    uint16_t* s_new = s_q + 8 * (D + QROW_PAD);       // fused step: the new token's rotated key [D], then its value [D]
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int g = lane >> 2, t = lane & 3;
@@ -815,8 +818,8 @@ decode_layer_kernel(SvlmAttendBatch b, int layer, const uint16_t* __restrict__ Q
                 if (h >= 8) continue;
                 const float x = h < G ? __bfloat162float(__ushort_as_bfloat16(qx[k])) : 0.f;
                 const float y = h < G ? __bfloat162float(__ushort_as_bfloat16(qy[k])) : 0.f;
-                s_q[h * D + pair] = __bfloat16_as_ushort(__float2bfloat16_rn(x * cs.x - y * cs.y));
-                s_q[h * D + pair + HALF] = __bfloat16_as_ushort(__float2bfloat16_rn(y * cs.x + x * cs.y));
+                s_q[h * (D + QROW_PAD) + pair] = __bfloat16_as_ushort(__float2bfloat16_rn(x * cs.x - y * cs.y));
+                s_q[h * (D + QROW_PAD) + pair + HALF] = __bfloat16_as_ushort(__float2bfloat16_rn(y * cs.x + x * cs.y));
             }
             if (prep_new) {
                 const float x = __bfloat162float(__ushort_as_bfloat16(kx)), y = __bfloat162float(__ushort_as_bfloat16(ky));
@@ -831,8 +834,8 @@ decode_layer_kernel(SvlmAttendBatch b, int layer, const uint16_t* __restrict__ Q
         unsigned qf[KSTEPS][2];   // B fragments of Q^T: (d = ks*16 + 2t.., head g)
 #pragma unroll
         for (int ks = 0; ks < KSTEPS; ++ks) {
-            qf[ks][0] = *reinterpret_cast<const unsigned*>(s_q + g * D + ks * 16 + 2 * t);
-            qf[ks][1] = *reinterpret_cast<const unsigned*>(s_q + g * D + ks * 16 + 2 * t + 8);
+            qf[ks][0] = *reinterpret_cast<const unsigned*>(s_q + g * (D + QROW_PAD) + ks * 16 + 2 * t);
+            qf[ks][1] = *reinterpret_cast<const unsigned*>(s_q + g * (D + QROW_PAD) + ks * 16 + 2 * t + 8);
         }
 
         const float scale = 1.4426950408889634f * rsqrtf((float)D);
@@ -1010,7 +1013,7 @@ decode_layer_kernel(SvlmAttendBatch b, int layer, const uint16_t* __restrict__ Q
 
 template <int D>
 constexpr size_t decode_layer_smem() {
-    return sizeof(LayShared) + 128 + (size_t)DEC_CWARPS * LAY_SLOTS * UNIT * D * 2 + 8 * D * 2 + 2 * D * 2;
+    return sizeof(LayShared) + 128 + (size_t)DEC_CWARPS * LAY_SLOTS * UNIT * D * 2 + 8 * (D + QROW_PAD) * 2 + 2 * D * 2;
 }
 static_assert(merge_bytes<128>() <= (size_t)DEC_CWARPS * LAY_SLOTS * UNIT * 128 * 2 && merge_bytes<64>() <= (size_t)DEC_CWARPS * LAY_SLOTS * UNIT * 64 * 2,
               "the merge slabs live in the warps' slots");
