@@ -107,7 +107,7 @@ class Cache:
         self._h = h
 
     def close(self):
-        if getattr(self, "_h", None):
+        if getattr(self, "_h", None) and _lib is not None:      # (at interpreter exit the module may already be torn down)
             _lib.svlm_cache_destroy(self._h)
             self._h = None
 

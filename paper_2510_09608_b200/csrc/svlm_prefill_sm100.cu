@@ -170,6 +170,18 @@ prefill_kernel(SvlmAttendBatch b, int layer0, int n_layers, const uint16_t* __re
     const int m0 = (blockIdx.x >> 1) * PF_ROWS;
     const int r_lo = m0 / G, r_hi = min(n_q - 1, (m0 + PF_ROWS - 1) / G);
 
+    // The CTA's query rows and positions are read a few microseconds from now, in four dependent rounds of loads:
+    // ask for their lines now, so that those rounds find them in L2 (one token's G heads are G * D * 2 contiguous bytes).
+    {
+        const int line_per_tok = (G * D * 2 + 127) / 128;
+        for (int i = threadIdx.x; i < (r_hi - r_lo + 1) * line_per_tok; i += PF_THREADS) {
+            const int tk = i / line_per_tok, ln = i % line_per_tok;
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char*>(Q + ((q_row0 + r_lo + tk) * q_heads + hk * G) * D) + ln * 128));
+        }
+        if (threadIdx.x < 32)
+            for (int i = threadIdx.x * 32; i < (r_hi - r_lo + 1) * (b.rope_mode == 0 ? 1 : 3); i += 32 * 32)
+                asm volatile("prefetch.global.L2 [%0];" ::"l"(q_pos + (p_row0 + r_lo) * (b.rope_mode == 0 ? 1 : 3) + i));
+    }
     const int n_tiles = min(vw.ctrl->n_tiles, PF_MAX_TILES);
     const long long gid_q0 = vw.ctrl->n_total - n_q;
     const long long shift = vw.ctrl->shift_total;
