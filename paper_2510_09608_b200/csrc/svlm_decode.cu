@@ -124,12 +124,18 @@ __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commi
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
-// Scratch layout per cache: arrival counters [layers*kv_heads] (zero between launches), then per
+// Scratch layout per cache: arrival counters [layers*kv_heads] (zero between launches) and the per-layer kernel's
+// two words per KV head (ws_head_words), then per
 // (layer in launch, kv head): splits records { o[8][D] bf16, m[8] f32, l[8] f32 }.  The
 // un-normalised partial outputs travel as bf16 (their error is of the size of the final rounding of
 // the output), which lets the combining CTA stage every record in shared memory in one round trip.
 template <int D>
 __host__ __device__ constexpr int rec_bytes() { return 8 * D * 2 + 64; }
+// Words in front of the records: the streaming kernel's arrival counters [layers * kv_heads], then the per-layer
+// kernel's pair (arrivals, base) per KV head; rounded up so that the records start on a 16-byte boundary.
+__host__ __device__ inline size_t ws_head_words(int layers, int kv_heads) {
+    return ((size_t)layers * kv_heads + 2 * (size_t)kv_heads + 3) & ~(size_t)3;
+}
 template <int D>
 __host__ __device__ constexpr int partial_floats() { return rec_bytes<D>() / 4; }
 
@@ -304,6 +310,156 @@ __device__ __forceinline__ void arrive_and_combine(int* s_last, unsigned* counte
     }
 }
 
+// The per-layer kernel's form of the same step.  One CTA pulling all the records of a KV head through its own
+// port to L2 and merging them with code that runs once per launch (instruction fetch, not arithmetic, sets its
+// pace) was the longest single piece of the layer-step, so the LAST `shares` CTAs to arrive split the output between
+// them, at most eight groups of eight output elements each: the arrival index a CTA draws from the counter says
+// which groups it combines.  The very last arriver starts at once; the others poll the counter (every warp by itself,
+// bounded by `wait_limit` polls) until all splits are counted.  All CTAs of the launch are resident together
+// (grid <= 2 CTAs per SM, and a programmatically launched successor only enters once every CTA here has passed
+// its launch trigger), so the wait is short; should it run out all the same, the CTA records SVLM_ERR_TIMEOUT and
+// leaves its groups unwritten.
+//
+// words[0] counts arrivals and is never set back: words[1] holds the count at which this launch started (`base`,
+// read by every CTA after the grid-dependency wait and handed in), and the last arriver moves it on by `splits`
+// for the next launch.  Nothing else writes it, every CTA has read it before it arrives, and the next launch
+// reads it only after this one has completed, so all CTAs of a launch see the same base and nobody has to
+// tidy up after the pollers.  The pieces of the records come straight from L2 into registers, coalesced: eight
+// lanes of a warp cover the (up to) eight groups of the CTA's share, which lie side by side in a record, the four
+// lane groups of the 7 warps take 28 records at a time, two rounds in flight (one record per lane with the lanes
+// 2112 bytes apart was 2 us slower: 32 cache lines per load instruction).  The four record lanes meet through
+// shuffles, the warps through `buf` (7 x 8 x 12 floats), and four threads per group write the result.  Called by
+// all DEC_THREADS threads after a __syncthreads() that follows the record's stores.  s_slot: shared word, on
+// return 1 + arrival rank from the end for a combining CTA, 0 otherwise.  stamp: trace hook (stations 8..10, 12, 13, 15).
+constexpr int DEC_WARPS = DEC_THREADS / 32;
+
+template <int D, typename Stamp>
+__device__ __forceinline__ void arrive_and_combine_shared(int* s_slot, unsigned* words, unsigned base, int splits,
+                                                          const unsigned char* parts, float* buf, int G, uint16_t* out_row0,
+                                                          unsigned wait_limit, int* status, Stamp stamp) {
+    constexpr int REC = rec_bytes<D>();
+    const int groups = G * (D / 8);                                         // groups of eight output elements
+    const int shares = min(splits, (groups + DEC_WARPS - 1) / DEC_WARPS);   // combining CTAs
+    const int per = (groups + shares - 1) / shares;                         // groups of one share
+    if (threadIdx.x == 0) {
+        stamp(8);
+        unsigned prev;
+        asm volatile("atom.add.acq_rel.gpu.global.u32 %0, [%1], 1;" : "=r"(prev) : "l"(words) : "memory");
+        const int share = splits - 1 - (int)(prev - base);   // 0 for the last arriver
+        if (share == 0) __stcg(words + 1, base + (unsigned)splits);
+        *s_slot = share < shares ? share + 1 : 0;
+        stamp(9);
+        if (share >= shares) stamp(13);
+    }
+    __syncthreads();
+    const int share = *s_slot - 1;
+    if (share < 0) return;
+    if (share > 0) {
+        bool complete = true;
+        for (unsigned polls = 0;; ++polls) {
+            if (polls >= wait_limit) { complete = false; break; }
+            unsigned v;
+            asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(words) : "memory");
+            if (v - base >= (unsigned)splits) break;
+        }
+        if (!__syncthreads_and(complete)) {
+            if (threadIdx.x == 0) atomicCAS(status, 0, -5);   // SVLM_ERR_TIMEOUT
+            return;
+        }
+    }
+    if (threadIdx.x == 0) stamp(10);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int gl = lane & 7, rl = lane >> 3;
+    float* slab = buf + (size_t)(warp * 8 + gl) * 12;   // [warp][group of the round][M, L, acc[8], pad]
+#pragma unroll 1
+    for (int g0 = 0; g0 < per; g0 += 8) {
+        const int grp = share * per + g0 + gl;
+        const bool valid = g0 + gl < per && grp < groups;
+        const int h = valid ? grp / (D / 8) : 0, d0 = valid ? (grp % (D / 8)) * 8 : 0;
+        const unsigned char* ml = parts + 8 * D * 2 + h * 4;
+        const unsigned char* ov = parts + (size_t)(h * D + d0) * 2;
+        float M = -INFINITY, L = 0.f;
+        float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+#pragma unroll 1
+        for (int r0 = warp * 4 + rl; r0 < splits; r0 += 2 * DEC_WARPS * 4) {
+            float mr[2], lr[2];
+            uint4 v[2];
+#pragma unroll
+            for (int k = 0; k < 2; ++k) {
+                const int r = r0 + k * DEC_WARPS * 4;
+                const size_t off = (size_t)(r < splits ? r : r0) * REC;
+                mr[k] = __ldcg(reinterpret_cast<const float*>(ml + off));
+                lr[k] = __ldcg(reinterpret_cast<const float*>(ml + off + 32));
+                v[k] = __ldcg(reinterpret_cast<const uint4*>(ov + off));
+                if (r >= splits || !valid) mr[k] = -INFINITY;   // weight 0
+            }
+            const float Mn = fmaxf(M, fmaxf(mr[0], mr[1]));
+            if (Mn > -INFINITY) {
+                const float resc = exp2f(M - Mn);             // M = -inf gives 0
+                L *= resc;
+#pragma unroll
+                for (int e = 0; e < 8; ++e) acc[e] *= resc;
+#pragma unroll
+                for (int k = 0; k < 2; ++k) {
+                    const float w = exp2f(mr[k] - Mn);
+                    L += lr[k] * w;
+                    acc[0] += __uint_as_float(v[k].x << 16) * w; acc[1] += __uint_as_float(v[k].x & 0xffff0000u) * w;
+                    acc[2] += __uint_as_float(v[k].y << 16) * w; acc[3] += __uint_as_float(v[k].y & 0xffff0000u) * w;
+                    acc[4] += __uint_as_float(v[k].z << 16) * w; acc[5] += __uint_as_float(v[k].z & 0xffff0000u) * w;
+                    acc[6] += __uint_as_float(v[k].w << 16) * w; acc[7] += __uint_as_float(v[k].w & 0xffff0000u) * w;
+                }
+                M = Mn;
+            }
+        }
+        if (threadIdx.x == 0) stamp(12);
+        // the four record lanes of a group meet: common maximum first, then the sums
+        const float Mw = fmaxf(fmaxf(M, __shfl_xor_sync(0xffffffffu, M, 8)),
+                               fmaxf(__shfl_xor_sync(0xffffffffu, M, 16), __shfl_xor_sync(0xffffffffu, M, 24)));
+        const float f = M > -INFINITY ? exp2f(M - Mw) : 0.f;
+        L *= f;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc[e] *= f;
+#pragma unroll
+        for (int sft = 8; sft < 32; sft <<= 1) {
+            L += __shfl_xor_sync(0xffffffffu, L, sft);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) acc[e] += __shfl_xor_sync(0xffffffffu, acc[e], sft);
+        }
+        if (rl == 0) {
+            *reinterpret_cast<float4*>(slab) = make_float4(Mw, L, acc[0], acc[1]);
+            *reinterpret_cast<float4*>(slab + 4) = make_float4(acc[2], acc[3], acc[4], acc[5]);
+            *reinterpret_cast<float2*>(slab + 8) = make_float2(acc[6], acc[7]);
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) stamp(15);
+        // the warps' shares of a group meet: four threads per group, two output elements each
+        if (threadIdx.x < 32) {
+            const int fg = lane >> 2, e2 = lane & 3;
+            const int fgrp = share * per + g0 + fg;
+            const float* sl = buf + (size_t)fg * 12;
+            float Ma = -INFINITY;
+#pragma unroll
+            for (int w = 0; w < DEC_WARPS; ++w) Ma = fmaxf(Ma, sl[w * 96]);
+            float La = 0.f, a0 = 0.f, a1 = 0.f;
+            if (Ma > -INFINITY)
+#pragma unroll
+                for (int w = 0; w < DEC_WARPS; ++w) {
+                    const float wt = exp2f(sl[w * 96] - Ma);
+                    const float2 a = *reinterpret_cast<const float2*>(sl + w * 96 + 2 + 2 * e2);
+                    La += sl[w * 96 + 1] * wt;
+                    a0 += a.x * wt;
+                    a1 += a.y * wt;
+                }
+            if (g0 + fg < per && fgrp < groups) {
+                const float inv = La > 0.f ? 1.f / La : 0.f;
+                const int fh = fgrp / (D / 8), fd = (fgrp % (D / 8)) * 8 + 2 * e2;
+                *reinterpret_cast<uint32_t*>(out_row0 + (size_t)fh * D + fd) = pack_bf16(a0 * inv, a1 * inv);
+            }
+        }
+        if (g0 + 8 < per) __syncthreads();   // the slabs are read before the next round writes them
+    }
+}
+
 // =============================== streaming kernel (several problems per launch) ===============================
 
 struct DecShared {
@@ -388,7 +544,7 @@ decode_stream_kernel(SvlmAttendBatch b, int layer0, int n_layers, const uint16_t
     const int q0 = (int)((long long)split * total_q / splits), q1 = (int)((long long)(split + 1) * total_q / splits);
     const size_t head_row0 = ((size_t)layer * b.kv_heads + hk) * b.n_slots;
     constexpr int REC = rec_bytes<D>();
-    unsigned char* ws_parts = reinterpret_cast<unsigned char*>(vw.ws + (((size_t)b.layers * b.kv_heads + 3) & ~(size_t)3));
+    unsigned char* ws_parts = reinterpret_cast<unsigned char*>(vw.ws + ws_head_words(b.layers, b.kv_heads));
     unsigned char* part = ws_parts + ((size_t)(li * b.kv_heads + hk) * splits + split) * REC;   // 16-byte aligned
 
     auto sub_valid = [&](int q, int& page, int& lo, int& hi) {
@@ -649,8 +805,10 @@ static_assert(merge_bytes<128>() <= (size_t)DEC_STAGES * 2 * SUB * 128 * 2 && me
 // =============================== per-layer kernel (one problem per launch) ===============================
 
 struct LayShared {
-    int last;
-    int pad[3];
+    int last;                          // 1 + the share of the final combine this CTA takes, 0: none
+    int wait_limit;                    // polls a waiting combiner may spend
+    int base;                          // the arrival counter's value when this launch started
+    int pad;
     unsigned tile_pk[DEC_MAX_TILES];   // page | lo << 16 | hi << 24
 };
 
@@ -708,6 +866,7 @@ decode_layer_kernel(SvlmAttendBatch b, int layer, const uint16_t* __restrict__ Q
         for (int o = 0; o < bytes; o += 128)
             asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char*>(p) + o));
     }
+    if (threadIdx.x == 0) sh.wait_limit = (int)min(__ldcg(&vw.ctrl->wait_limit), 0x7fffffffu);
     const long long shift = __ldcg(&vw.ctrl->shift_total);
     // the new token of a fused step: where it lives and whether it is still stored there
     int new_slot = -1;
@@ -725,8 +884,9 @@ decode_layer_kernel(SvlmAttendBatch b, int layer, const uint16_t* __restrict__ Q
     const int n_rounds = (n_units + GROUP - 1) / GROUP;
     const size_t head_row0 = ((size_t)layer * b.kv_heads + hk) * b.n_slots;
     constexpr int REC = rec_bytes<D>();
-    unsigned char* ws_parts = reinterpret_cast<unsigned char*>(vw.ws + (((size_t)b.layers * b.kv_heads + 3) & ~(size_t)3));
+    unsigned char* ws_parts = reinterpret_cast<unsigned char*>(vw.ws + ws_head_words(b.layers, b.kv_heads));
     unsigned char* part = ws_parts + ((size_t)hk * splits + split) * REC;   // 16-byte aligned
+    unsigned* lay_words = reinterpret_cast<unsigned*>(vw.ws) + (size_t)b.layers * b.kv_heads + 2 * hk;   // arrivals, base
 
     if (consumer) {
         const uint16_t* Kh = vw.K + head_row0 * D;
@@ -793,6 +953,8 @@ decode_layer_kernel(SvlmAttendBatch b, int layer, const uint16_t* __restrict__ Q
             const float2 cs = svlm_rope_cs(tab, HALF, pair, cpos, b.theta[pair]);
             if (new_slot >= 0 && early_loads) pdl_wait();
             if (threadIdx.x == 0) STAMP(3);          // the previous kernel has completed
+            unsigned base = 0;                       // the arrival counter's start value (same round trip as the query)
+            if (threadIdx.x == 0) base = __ldcg(lay_words + 1);
             constexpr int HSTEP = (DEC_CWARPS * 32) / HALF, HN = (8 + HSTEP - 1) / HSTEP;   // heads per thread
             uint16_t qx[HN], qy[HN];
             // fused step: the new token's key and value rows come in with the query (same round trip); the key is
@@ -828,6 +990,7 @@ decode_layer_kernel(SvlmAttendBatch b, int layer, const uint16_t* __restrict__ Q
                 s_new[D + pair] = vx;
                 s_new[D + pair + HALF] = vy;
             }
+            if (threadIdx.x == 0) sh.base = (int)base;
         }
         asm volatile("bar.sync 1, %0;" ::"n"(DEC_CWARPS * 32));   // consumer warps only
         if (threadIdx.x == 0) STAMP(4);              // rotated query in shared memory
@@ -1003,8 +1166,8 @@ decode_layer_kernel(SvlmAttendBatch b, int layer, const uint16_t* __restrict__ Q
 #else
     auto stamp = [](int) {};
 #endif
-    arrive_and_combine<D, RING_BYTES>(&sh.last, reinterpret_cast<unsigned*>(vw.ws) + hk, splits,
-                                      ws_parts + (size_t)hk * splits * REC, ring, G, out + (size_t)hk * G * D, false, stamp);
+    arrive_and_combine_shared<D>(&sh.last, lay_words, (unsigned)sh.base, splits, ws_parts + (size_t)hk * splits * REC,
+                                 reinterpret_cast<float*>(ring), G, out + (size_t)hk * G * D, (unsigned)sh.wait_limit, const_cast<int*>(&vw.ctrl->status), stamp);
 #ifdef SVLM_DECODE_TRACE
     __syncthreads();
     if (threadIdx.x == 0 && sh.last) { STAMP(11); STAMP(13); }   // output written; leaving
@@ -1023,8 +1186,10 @@ static_assert(merge_bytes<128>() <= (size_t)DEC_CWARPS * LAY_SLOTS * UNIT * 128 
 // Scratch floats needed per cache for `splits` splits (all layers at once is the largest launch).
 size_t svlm_decode_ws_floats(int layers, int kv_heads, int head_dim, int splits) {
     const size_t pf = head_dim == 128 ? partial_floats<128>() : partial_floats<64>();
-    return (((size_t)layers * kv_heads + 3) & ~(size_t)3) + (size_t)layers * kv_heads * splits * pf;
+    return ws_head_words(layers, kv_heads) + (size_t)layers * kv_heads * splits * pf;
 }
+
+size_t svlm_decode_ws_head_floats(int layers, int kv_heads) { return ws_head_words(layers, kv_heads); }
 
 bool svlm_decode_supported(int n_pages) { return n_pages <= DEC_MAX_TILES; }
 

@@ -44,6 +44,8 @@ void svlm_launch_attend_simple(const SvlmAttendBatch& b, int layer0, int n_layer
 
 // split-KV decode, n_q = 1 (svlm_decode.cu)
 size_t svlm_decode_ws_floats(int layers_in_launch, int kv_heads, int head_dim, int splits);
+// the words in front of the records (arrival counters and the like) for a cache of `layers` layers
+size_t svlm_decode_ws_head_floats(int layers, int kv_heads);
 int svlm_decode_splits(int n_pages, int kv_heads, int problems);
 // The kernel keeps the list of active pages in shared memory: caches with more pages take the general kernel.
 bool svlm_decode_supported(int n_pages);

@@ -79,12 +79,31 @@ def test_batched_decode_gives_up_counter_returns_to_zero():
         for i, s in enumerate(sides):
             s._give_values_to_ref(0)
             assert_close(s._stats(out[i], s.ref.attend(0, s.stream.q(0, s.last[0]), s.last[2])))
-    # one cache, one layer: that kernel loads with cp.async and has no bounded wait to run out
+
+
+def test_layer_decode_waiting_combiners_give_up_counter_returns_to_zero():
+    """The per-layer split-KV kernel (one cache, one layer): its copies are cp.async and cannot time out, but the last
+    few CTAs to arrive share the final combine and all but the very last of them poll the arrival counter.  With the
+    limit at 0 they give up before their first poll: time-out recorded, their shares of the output unwritten, and the
+    counter (arrivals and finished waiters in its two halves) back at zero whichever CTA completed it."""
+    from harness import assert_close, bits_to_dev, dev_to_f64
+    from paper_2510_09608_b200 import binding
+    wl = _small(True)
     one = _filled(wl, stream_id=5)
     one.append_decode_token()
+    gids, _, pos = one.last
+    Q = bits_to_dev(one.stream.q(0, gids))
+    qp = torch.from_numpy(np.ascontiguousarray(pos)).cuda()
     one.cache.debug_set_wait_limit(0)
-    assert_close(one.attend(0))
-    assert one.cache.status() == binding.OK
+    for _ in range(3):
+        one.cache.attend(0, Q, qp)
+    assert one.cache.status() == binding.ERR_TIMEOUT
+    one.cache.debug_set_wait_limit(1 << 20)
+    one._give_values_to_ref(0)
+    want = one.ref.attend(0, one.stream.q(0, gids), pos)
+    for _ in range(2):
+        assert_close(one._stats(dev_to_f64(one.cache.attend(0, Q, qp)), want))
+    assert one.cache.status() == binding.ERR_TIMEOUT        # sticky
 
 
 def test_projection_gives_up_and_recovers():
