@@ -1004,8 +1004,8 @@ def bench_drift(args, wl, base, peaks, rank, world, local):
 TRACE_STATIONS = {0: "kernel entry", 1: "page list in shared memory", 2: "first round's copies issued",
                   3: "previous kernel complete (dependency wait returns)", 4: "rotated query in shared memory",
                   5: "warp 1 has its keys", 14: "warp 1: scores and softmax done", 6: "warp 1 through with its units",
-                  7: "all consumer warps through", 8: "CTA's record written", 9: "arrival counted",
-                  10: "combining CTA: all splits counted", 12: "combining CTA: its pieces of the records in registers",
+                  7: "all consumer warps through", 8: "CTA's record on its way (tagged stores issued)",
+                  12: "combining CTA: its pieces of every split's record in registers",
                   15: "combining CTA: warps' sums exchanged", 11: "combining CTA: output written", 13: "CTA leaves"}
 
 

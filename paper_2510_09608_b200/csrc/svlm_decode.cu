@@ -124,20 +124,39 @@ __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commi
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
-// Scratch layout per cache: arrival counters [layers*kv_heads] (zero between launches) and the per-layer kernel's
-// two words per KV head (ws_head_words), then per
+// Scratch layout per cache: arrival counters [layers*kv_heads] (zero between launches), then per
 // (layer in launch, kv head): splits records { o[8][D] bf16, m[8] f32, l[8] f32 }.  The
 // un-normalised partial outputs travel as bf16 (their error is of the size of the final rounding of
 // the output), which lets the combining CTA stage every record in shared memory in one round trip.
 template <int D>
 __host__ __device__ constexpr int rec_bytes() { return 8 * D * 2 + 64; }
-// Words in front of the records: the streaming kernel's arrival counters [layers * kv_heads], then the per-layer
-// kernel's pair (arrivals, base) per KV head; rounded up so that the records start on a 16-byte boundary.
+// Words in front of the records: the arrival counters [layers * kv_heads], rounded up so that the records start
+// on a 16-byte boundary.
 __host__ __device__ inline size_t ws_head_words(int layers, int kv_heads) {
-    return ((size_t)layers * kv_heads + 2 * (size_t)kv_heads + 3) & ~(size_t)3;
+    return ((size_t)layers * kv_heads + 3) & ~(size_t)3;
 }
+
+// The per-layer kernel's records live in an area of their own and carry a tag in every 64-bit word
+// { payload, tag } (the payload: two bf16 partial outputs, or a head's maximum or sum as fp32): a reader that
+// finds this launch's tag in a word has that word's payload, since an aligned 64-bit access is single-copy
+// atomic.  No fence, no counter and no second round trip stand between a CTA's stores and the combining CTAs'
+// loads.  Layout of the area: one epoch word per KV head (rounded up to 128 bytes), then per (KV head, split) a
+// record { o[8][D] as 4 D words of 8 bytes, then per head (m, tag), (l, tag) }.  Nothing but tagged words is
+// ever written to the record part, the tag of a launch is its KV head's epoch + 1 and the epoch goes up by one
+// per launch, so a word left by an earlier launch never carries the current tag.
+template <int D>
+__host__ __device__ constexpr int ll_rec_bytes() { return 8 * D * 4 + 8 * 16; }
+__host__ __device__ inline size_t ll_head_bytes(int kv_heads) { return ((size_t)kv_heads * 4 + 127) & ~(size_t)127; }
 template <int D>
 __host__ __device__ constexpr int partial_floats() { return rec_bytes<D>() / 4; }
+
+__device__ __forceinline__ void st_tagged2(void* p, unsigned a, unsigned b, unsigned tag) {
+    const unsigned long long hi = (unsigned long long)tag << 32;
+    asm volatile("st.relaxed.gpu.global.v2.b64 [%0], {%1, %2};" ::"l"(p), "l"(hi | a), "l"(hi | b) : "memory");
+}
+__device__ __forceinline__ void ld_tagged2(const void* p, unsigned long long& a, unsigned long long& b) {
+    asm volatile("ld.relaxed.gpu.global.v2.b64 {%0, %1}, [%2];" : "=l"(a), "=l"(b) : "l"(p) : "memory");
+}
 
 // ---- the part both kernels share: from the consumer warps' accumulators to the output -----------------------
 
@@ -145,9 +164,10 @@ __host__ __device__ constexpr int partial_floats() { return rec_bytes<D>() / 4; 
 // running maximum and sum of heads 2t, 2t+1) through `buf` and store of the CTA's record at `part`.  Called by
 // the consumer warps only.  One slab [8 heads][D + 4] of fp32 per warp: with the padded row the 32 lanes of a
 // store (4 head pairs x 8 dims) fall into 32 different banks.
-template <int D, typename Stamp>
+// TAGGED: the record goes out in the per-layer kernel's tagged format (ll_rec_bytes).
+template <int D, bool TAGGED, typename Stamp>
 __device__ __forceinline__ void cta_merge_and_record(const float (&o)[D / 16][4], const float (&m)[2], const float (&l)[2],
-                                                     float* buf, unsigned char* part, Stamp stamp) {
+                                                     float* buf, unsigned char* part, unsigned tag, Stamp stamp) {
     constexpr int MROW = D + MERGE_PAD, DBLK = D / 16;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, g = lane >> 2, t = lane & 3;
     float* s_o = buf;                                     // [warp][8 heads][MROW]
@@ -189,7 +209,12 @@ __device__ __forceinline__ void cta_merge_and_record(const float (&o)[D / 16][4]
         uint4 pk;
         pk.x = pack_bf16(acc[0], acc[1]); pk.y = pack_bf16(acc[2], acc[3]);
         pk.z = pack_bf16(acc[4], acc[5]); pk.w = pack_bf16(acc[6], acc[7]);
-        *reinterpret_cast<uint4*>(part + (size_t)(h * D + d0) * 2) = pk;
+        if constexpr (TAGGED) {
+            st_tagged2(part + (size_t)(h * D + d0) * 4, pk.x, pk.y, tag);
+            st_tagged2(part + (size_t)(h * D + d0) * 4 + 16, pk.z, pk.w, tag);
+        } else {
+            *reinterpret_cast<uint4*>(part + (size_t)(h * D + d0) * 2) = pk;
+        }
     } else if (ct < D + 8) {
         const int h = ct - D;
         float M = -INFINITY, L = 0.f;
@@ -198,9 +223,13 @@ __device__ __forceinline__ void cta_merge_and_record(const float (&o)[D / 16][4]
         if (M > -INFINITY)
 #pragma unroll
             for (int w = 0; w < DEC_CWARPS; ++w) L += s_l[w * 8 + h] * exp2f(s_m[w * 8 + h] - M);
-        float* ml = reinterpret_cast<float*>(part + 8 * D * 2);
-        ml[h] = M;
-        ml[8 + h] = L;
+        if constexpr (TAGGED) {
+            st_tagged2(part + 8 * D * 4 + h * 16, __float_as_uint(M), __float_as_uint(L), tag);
+        } else {
+            float* ml = reinterpret_cast<float*>(part + 8 * D * 2);
+            ml[h] = M;
+            ml[8 + h] = L;
+        }
     }
 }
 
@@ -312,101 +341,95 @@ __device__ __forceinline__ void arrive_and_combine(int* s_last, unsigned* counte
 
 // The per-layer kernel's form of the same step.  One CTA pulling all the records of a KV head through its own
 // port to L2 and merging them with code that runs once per launch (instruction fetch, not arithmetic, sets its
-// pace) was the longest single piece of the layer-step, so the LAST `shares` CTAs to arrive split the output between
-// them, at most eight groups of eight output elements each: the arrival index a CTA draws from the counter says
-// which groups it combines.  The very last arriver starts at once; the others poll the counter (every warp by itself,
-// bounded by `wait_limit` polls) until all splits are counted.  All CTAs of the launch are resident together
-// (grid <= 2 CTAs per SM, and a programmatically launched successor only enters once every CTA here has passed
-// its launch trigger), so the wait is short; should it run out all the same, the CTA records SVLM_ERR_TIMEOUT and
-// leaves its groups unwritten.
+// pace) was the longest single piece of the layer-step, and the release fence plus the arrival atomic in front of
+// it the next longest.  Here the first `shares` splits of a KV head split the output between them, at most eight
+// groups of eight output elements each, and read their pieces of all the records in the tagged format (see
+// ll_rec_bytes): a word that carries this launch's tag is that record's word.  Words that do not yet are read
+// again, at most `wait_limit` times per thread; then the CTA records SVLM_ERR_TIMEOUT and writes whatever it has
+// (limit 0: without a first try).  All CTAs of the launch are resident together (grid <= 2 CTAs per SM, and a
+// programmatically launched successor only enters once every CTA here has passed its launch trigger), so the
+// wait is for stragglers only.
 //
-// words[0] counts arrivals and is never set back: words[1] holds the count at which this launch started (`base`,
-// read by every CTA after the grid-dependency wait and handed in), and the last arriver moves it on by `splits`
-// for the next launch.  Nothing else writes it, every CTA has read it before it arrives, and the next launch
-// reads it only after this one has completed, so all CTAs of a launch see the same base and nobody has to
-// tidy up after the pollers.  The pieces of the records come straight from L2 into registers, coalesced: eight
-// lanes of a warp cover the (up to) eight groups of the CTA's share, which lie side by side in a record, the four
-// lane groups of the 7 warps take 28 records at a time, two rounds in flight (one record per lane with the lanes
-// 2112 bytes apart was 2 us slower: 32 cache lines per load instruction).  The four record lanes meet through
-// shuffles, the warps through `buf` (7 x 8 x 12 floats), and four threads per group write the result.  Called by
-// all DEC_THREADS threads after a __syncthreads() that follows the record's stores.  s_slot: shared word, on
-// return 1 + arrival rank from the end for a combining CTA, 0 otherwise.  stamp: trace hook (stations 8..10, 12, 13, 15).
+// The loads are coalesced: eight lanes of a warp cover the (up to) eight groups of the CTA's share, which lie side
+// by side in a record, the four lane groups of the 7 warps take 28 records at a time, two rounds in flight (one
+// record per lane with the lanes a record apart was 2 us slower: 32 cache lines per load instruction).  The four
+// record lanes meet through shuffles, the warps through `buf` (7 x 8 x 12 floats), and four threads per group
+// write the result.  Split 0, which by then has seen every split's record and therefore knows that every CTA of
+// the KV head has read the epoch, moves the epoch on for the next launch.  Called by all DEC_THREADS threads of the
+// first `shares` splits after a __syncthreads() that follows their last use of `buf`.
+// stamp: trace hook (stations 12, 15).
 constexpr int DEC_WARPS = DEC_THREADS / 32;
 
+__host__ __device__ inline int combine_shares(int groups, int splits) {
+    const int want = (groups + DEC_WARPS - 1) / DEC_WARPS;
+    return want < splits ? want : splits;
+}
+
 template <int D, typename Stamp>
-__device__ __forceinline__ void arrive_and_combine_shared(int* s_slot, unsigned* words, unsigned base, int splits,
-                                                          const unsigned char* parts, float* buf, int G, uint16_t* out_row0,
-                                                          unsigned wait_limit, int* status, Stamp stamp) {
-    constexpr int REC = rec_bytes<D>();
-    const int groups = G * (D / 8);                                         // groups of eight output elements
-    const int shares = min(splits, (groups + DEC_WARPS - 1) / DEC_WARPS);   // combining CTAs
-    const int per = (groups + shares - 1) / shares;                         // groups of one share
-    if (threadIdx.x == 0) {
-        stamp(8);
-        unsigned prev;
-        asm volatile("atom.add.acq_rel.gpu.global.u32 %0, [%1], 1;" : "=r"(prev) : "l"(words) : "memory");
-        const int share = splits - 1 - (int)(prev - base);   // 0 for the last arriver
-        if (share == 0) __stcg(words + 1, base + (unsigned)splits);
-        *s_slot = share < shares ? share + 1 : 0;
-        stamp(9);
-        if (share >= shares) stamp(13);
-    }
-    __syncthreads();
-    const int share = *s_slot - 1;
-    if (share < 0) return;
-    if (share > 0) {
-        bool complete = true;
-        for (unsigned polls = 0;; ++polls) {
-            if (polls >= wait_limit) { complete = false; break; }
-            unsigned v;
-            asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(words) : "memory");
-            if (v - base >= (unsigned)splits) break;
-        }
-        if (!__syncthreads_and(complete)) {
-            if (threadIdx.x == 0) atomicCAS(status, 0, -5);   // SVLM_ERR_TIMEOUT
-            return;
-        }
-    }
-    if (threadIdx.x == 0) stamp(10);
+__device__ __forceinline__ void combine_tagged(int share, int shares, int splits, const unsigned char* parts, unsigned tag,
+                                               unsigned* epoch, float* buf, int G, uint16_t* out_row0, unsigned wait_limit,
+                                               int* status, Stamp stamp) {
+    constexpr int REC = ll_rec_bytes<D>();
+    const int groups = G * (D / 8);                          // groups of eight output elements
+    const int per = (groups + shares - 1) / shares;          // groups of one share
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int gl = lane & 7, rl = lane >> 3;
-    float* slab = buf + (size_t)(warp * 8 + gl) * 12;   // [warp][group of the round][M, L, acc[8], pad]
+    float* slab = buf + (size_t)(warp * 8 + gl) * 12;        // [warp][group of the round][M, L, acc[8], pad]
+    bool timed_out = false;
 #pragma unroll 1
     for (int g0 = 0; g0 < per; g0 += 8) {
         const int grp = share * per + g0 + gl;
         const bool valid = g0 + gl < per && grp < groups;
         const int h = valid ? grp / (D / 8) : 0, d0 = valid ? (grp % (D / 8)) * 8 : 0;
-        const unsigned char* ml = parts + 8 * D * 2 + h * 4;
-        const unsigned char* ov = parts + (size_t)(h * D + d0) * 2;
+        const unsigned char* ml = parts + 8 * D * 4 + h * 16;
+        const unsigned char* ov = parts + (size_t)(h * D + d0) * 4;
         float M = -INFINITY, L = 0.f;
         float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
 #pragma unroll 1
         for (int r0 = warp * 4 + rl; r0 < splits; r0 += 2 * DEC_WARPS * 4) {
-            float mr[2], lr[2];
-            uint4 v[2];
+            unsigned long long w[2][6];                      // per record: o words 0..3, (m, tag), (l, tag)
+            bool want[2];
 #pragma unroll
-            for (int k = 0; k < 2; ++k) {
-                const int r = r0 + k * DEC_WARPS * 4;
-                const size_t off = (size_t)(r < splits ? r : r0) * REC;
-                mr[k] = __ldcg(reinterpret_cast<const float*>(ml + off));
-                lr[k] = __ldcg(reinterpret_cast<const float*>(ml + off + 32));
-                v[k] = __ldcg(reinterpret_cast<const uint4*>(ov + off));
-                if (r >= splits || !valid) mr[k] = -INFINITY;   // weight 0
+            for (int k = 0; k < 2; ++k) want[k] = valid && r0 + k * DEC_WARPS * 4 < splits;
+            for (unsigned polls = 0;; ++polls) {
+                if (polls >= wait_limit) { timed_out = true; break; }
+                bool ok = true;
+#pragma unroll
+                for (int k = 0; k < 2; ++k) {
+                    if (!want[k]) continue;
+                    const size_t off = (size_t)(r0 + k * DEC_WARPS * 4) * REC;
+                    ld_tagged2(ov + off, w[k][0], w[k][1]);
+                    ld_tagged2(ov + off + 16, w[k][2], w[k][3]);
+                    ld_tagged2(ml + off, w[k][4], w[k][5]);
+                }
+#pragma unroll
+                for (int k = 0; k < 2; ++k) {
+                    if (!want[k]) continue;
+#pragma unroll
+                    for (int i = 0; i < 6; ++i) ok = ok && (unsigned)(w[k][i] >> 32) == tag;
+                }
+                if (ok) break;
             }
+            float mr[2];
+#pragma unroll
+            for (int k = 0; k < 2; ++k) mr[k] = want[k] && !timed_out ? __uint_as_float((unsigned)w[k][4]) : -INFINITY;   // else weight 0
             const float Mn = fmaxf(M, fmaxf(mr[0], mr[1]));
             if (Mn > -INFINITY) {
-                const float resc = exp2f(M - Mn);             // M = -inf gives 0
+                const float resc = exp2f(M - Mn);            // M = -inf gives 0
                 L *= resc;
 #pragma unroll
                 for (int e = 0; e < 8; ++e) acc[e] *= resc;
 #pragma unroll
                 for (int k = 0; k < 2; ++k) {
-                    const float w = exp2f(mr[k] - Mn);
-                    L += lr[k] * w;
-                    acc[0] += __uint_as_float(v[k].x << 16) * w; acc[1] += __uint_as_float(v[k].x & 0xffff0000u) * w;
-                    acc[2] += __uint_as_float(v[k].y << 16) * w; acc[3] += __uint_as_float(v[k].y & 0xffff0000u) * w;
-                    acc[4] += __uint_as_float(v[k].z << 16) * w; acc[5] += __uint_as_float(v[k].z & 0xffff0000u) * w;
-                    acc[6] += __uint_as_float(v[k].w << 16) * w; acc[7] += __uint_as_float(v[k].w & 0xffff0000u) * w;
+                    if (mr[k] == -INFINITY) continue;
+                    const float wt = exp2f(mr[k] - Mn);
+                    L += __uint_as_float((unsigned)w[k][5]) * wt;
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const unsigned pr = (unsigned)w[k][i];
+                        acc[2 * i] += __uint_as_float(pr << 16) * wt;
+                        acc[2 * i + 1] += __uint_as_float(pr & 0xffff0000u) * wt;
+                    }
                 }
                 M = Mn;
             }
@@ -439,14 +462,14 @@ __device__ __forceinline__ void arrive_and_combine_shared(int* s_slot, unsigned*
             const float* sl = buf + (size_t)fg * 12;
             float Ma = -INFINITY;
 #pragma unroll
-            for (int w = 0; w < DEC_WARPS; ++w) Ma = fmaxf(Ma, sl[w * 96]);
+            for (int wp = 0; wp < DEC_WARPS; ++wp) Ma = fmaxf(Ma, sl[wp * 96]);
             float La = 0.f, a0 = 0.f, a1 = 0.f;
             if (Ma > -INFINITY)
 #pragma unroll
-                for (int w = 0; w < DEC_WARPS; ++w) {
-                    const float wt = exp2f(sl[w * 96] - Ma);
-                    const float2 a = *reinterpret_cast<const float2*>(sl + w * 96 + 2 + 2 * e2);
-                    La += sl[w * 96 + 1] * wt;
+                for (int wp = 0; wp < DEC_WARPS; ++wp) {
+                    const float wt = exp2f(sl[wp * 96] - Ma);
+                    const float2 a = *reinterpret_cast<const float2*>(sl + wp * 96 + 2 + 2 * e2);
+                    La += sl[wp * 96 + 1] * wt;
                     a0 += a.x * wt;
                     a1 += a.y * wt;
                 }
@@ -458,6 +481,8 @@ __device__ __forceinline__ void arrive_and_combine_shared(int* s_slot, unsigned*
         }
         if (g0 + 8 < per) __syncthreads();   // the slabs are read before the next round writes them
     }
+    if (share == 0 && threadIdx.x == 0) __stcg(epoch, tag);
+    if (timed_out) atomicCAS(status, 0, -5);   // SVLM_ERR_TIMEOUT
 }
 
 // =============================== streaming kernel (several problems per launch) ===============================
@@ -775,7 +800,7 @@ decode_stream_kernel(SvlmAttendBatch b, int layer0, int n_layers, const uint16_t
             l[1] += __shfl_xor_sync(0xffffffffu, l[1], sft);
         }
         // the ring is free once all consumer warps are here (the merge waits for that)
-        cta_merge_and_record<D>(o, m, l, reinterpret_cast<float*>(ring), part, [](int) {});
+        cta_merge_and_record<D, false>(o, m, l, reinterpret_cast<float*>(ring), part, 0u, [](int) {});
     }
 
     // ---- last CTA of this (cache, layer, kv head) combines the splits -----------------------------
@@ -805,10 +830,9 @@ static_assert(merge_bytes<128>() <= (size_t)DEC_STAGES * 2 * SUB * 128 * 2 && me
 // =============================== per-layer kernel (one problem per launch) ===============================
 
 struct LayShared {
-    int last;                          // 1 + the share of the final combine this CTA takes, 0: none
-    int wait_limit;                    // polls a waiting combiner may spend
-    int base;                          // the arrival counter's value when this launch started
-    int pad;
+    int tag;                           // this launch's tag of the records' words
+    int wait_limit;                    // times a combining thread may read a word again
+    int pad[2];
     unsigned tile_pk[DEC_MAX_TILES];   // page | lo << 16 | hi << 24
 };
 
@@ -822,7 +846,7 @@ template <int D>
 __global__ void __launch_bounds__(DEC_THREADS, 2)
 decode_layer_kernel(SvlmAttendBatch b, int layer, const uint16_t* __restrict__ Q, const int* __restrict__ q_pos, int q_heads,
                     uint16_t* __restrict__ out, int splits, const uint16_t* __restrict__ Knew,
-                    const uint16_t* __restrict__ Vnew, int early_loads TRACE_PARAM) {
+                    const uint16_t* __restrict__ Vnew, int early_loads, unsigned char* __restrict__ records TRACE_PARAM) {
     if (threadIdx.x == 0) STAMP(0);                  // kernel entry
     constexpr int CH = D / 8;                        // 16-byte chunks per row
     constexpr int ITEM_BYTES = UNIT * D * 2;         // K or V of one unit
@@ -883,10 +907,10 @@ decode_layer_kernel(SvlmAttendBatch b, int layer, const uint16_t* __restrict__ Q
     const int n_units = u1 - u0;
     const int n_rounds = (n_units + GROUP - 1) / GROUP;
     const size_t head_row0 = ((size_t)layer * b.kv_heads + hk) * b.n_slots;
-    constexpr int REC = rec_bytes<D>();
-    unsigned char* ws_parts = reinterpret_cast<unsigned char*>(vw.ws + ws_head_words(b.layers, b.kv_heads));
-    unsigned char* part = ws_parts + ((size_t)hk * splits + split) * REC;   // 16-byte aligned
-    unsigned* lay_words = reinterpret_cast<unsigned*>(vw.ws) + (size_t)b.layers * b.kv_heads + 2 * hk;   // arrivals, base
+    constexpr int REC = ll_rec_bytes<D>();
+    unsigned* epoch = reinterpret_cast<unsigned*>(records) + hk;
+    unsigned char* ws_parts = records + ll_head_bytes(b.kv_heads) + (size_t)hk * splits * REC;   // this KV head's records
+    unsigned char* part = ws_parts + (size_t)split * REC;                                       // 16-byte aligned
 
     if (consumer) {
         const uint16_t* Kh = vw.K + head_row0 * D;
@@ -953,8 +977,8 @@ decode_layer_kernel(SvlmAttendBatch b, int layer, const uint16_t* __restrict__ Q
             const float2 cs = svlm_rope_cs(tab, HALF, pair, cpos, b.theta[pair]);
             if (new_slot >= 0 && early_loads) pdl_wait();
             if (threadIdx.x == 0) STAMP(3);          // the previous kernel has completed
-            unsigned base = 0;                       // the arrival counter's start value (same round trip as the query)
-            if (threadIdx.x == 0) base = __ldcg(lay_words + 1);
+            unsigned ep = 0;                         // the KV head's epoch (same round trip as the query)
+            if (threadIdx.x == 0) ep = __ldcg(epoch);
             constexpr int HSTEP = (DEC_CWARPS * 32) / HALF, HN = (8 + HSTEP - 1) / HSTEP;   // heads per thread
             uint16_t qx[HN], qy[HN];
             // fused step: the new token's key and value rows come in with the query (same round trip); the key is
@@ -990,7 +1014,7 @@ decode_layer_kernel(SvlmAttendBatch b, int layer, const uint16_t* __restrict__ Q
                 s_new[D + pair] = vx;
                 s_new[D + pair + HALF] = vy;
             }
-            if (threadIdx.x == 0) sh.base = (int)base;
+            if (threadIdx.x == 0) sh.tag = (int)(ep + 1);
         }
         asm volatile("bar.sync 1, %0;" ::"n"(DEC_CWARPS * 32));   // consumer warps only
         if (threadIdx.x == 0) STAMP(4);              // rotated query in shared memory
@@ -1155,22 +1179,27 @@ decode_layer_kernel(SvlmAttendBatch b, int layer, const uint16_t* __restrict__ Q
 #else
         auto stamp7 = [](int) {};
 #endif
-        cta_merge_and_record<D>(o, m, l, reinterpret_cast<float*>(ring), part, stamp7);
+        cta_merge_and_record<D, true>(o, m, l, reinterpret_cast<float*>(ring), part, (unsigned)sh.tag, stamp7);
     }
 
-    // ---- last CTA of this KV head combines the splits -----------------------------
-    __syncthreads();
-    // The barrier above ordered every thread's partial-result stores before thread 0's release.
+    // ---- the first splits of this KV head combine all the splits' records -----------------------------
+    __syncthreads();                                  // the merge slabs in `ring` are read
+    if (threadIdx.x == 0) STAMP(8);                   // the CTA's record is on its way
+    const int shares = combine_shares(G * (D / 8), splits);
+    if (split >= shares) {
+        if (threadIdx.x == 0) STAMP(13);
+        return;
+    }
 #ifdef SVLM_DECODE_TRACE
     auto stamp = [&](int i) { STAMP(i); };
 #else
     auto stamp = [](int) {};
 #endif
-    arrive_and_combine_shared<D>(&sh.last, lay_words, (unsigned)sh.base, splits, ws_parts + (size_t)hk * splits * REC,
-                                 reinterpret_cast<float*>(ring), G, out + (size_t)hk * G * D, (unsigned)sh.wait_limit, const_cast<int*>(&vw.ctrl->status), stamp);
+    combine_tagged<D>(split, shares, splits, ws_parts, (unsigned)sh.tag, epoch, reinterpret_cast<float*>(ring), G,
+                      out + (size_t)hk * G * D, (unsigned)sh.wait_limit, const_cast<int*>(&vw.ctrl->status), stamp);
 #ifdef SVLM_DECODE_TRACE
     __syncthreads();
-    if (threadIdx.x == 0 && sh.last) { STAMP(11); STAMP(13); }   // output written; leaving
+    if (threadIdx.x == 0) { STAMP(11); STAMP(13); }   // output written; leaving
 #endif
 }
 
@@ -1189,7 +1218,10 @@ size_t svlm_decode_ws_floats(int layers, int kv_heads, int head_dim, int splits)
     return ws_head_words(layers, kv_heads) + (size_t)layers * kv_heads * splits * pf;
 }
 
-size_t svlm_decode_ws_head_floats(int layers, int kv_heads) { return ws_head_words(layers, kv_heads); }
+// Bytes of the per-layer kernel's area of tagged records (zero-filled at allocation, never written by anything else).
+size_t svlm_decode_tagged_bytes(int kv_heads, int head_dim, int splits) {
+    return ll_head_bytes(kv_heads) + (size_t)kv_heads * splits * (head_dim == 128 ? ll_rec_bytes<128>() : ll_rec_bytes<64>());
+}
 
 bool svlm_decode_supported(int n_pages) { return n_pages <= DEC_MAX_TILES; }
 
@@ -1205,7 +1237,7 @@ int svlm_decode_splits(int n_pages, int kv_heads, int problems) {
 
 cudaError_t svlm_launch_decode(const SvlmAttendBatch& b, int layer0, int n_layers, const void* Q, const int* q_pos,
                                int q_heads, void* out, int splits, const void* Knew, const void* Vnew, int early_loads,
-                               cudaStream_t st) {
+                               void* tagged, cudaStream_t st) {
     const int problems = b.n_caches * n_layers;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(splits, b.kv_heads, problems);
@@ -1221,7 +1253,7 @@ cudaError_t svlm_launch_decode(const SvlmAttendBatch& b, int layer0, int n_layer
     const uint16_t* Kn = (const uint16_t*)Knew;
     const uint16_t* Vn = (const uint16_t*)Vnew;
     cudaError_t e;
-    if (problems == 1) {
+    if (problems == 1 && tagged) {
 #ifdef SVLM_DECODE_TRACE
         int trace_idx = -1;
         if (g_decode_trace_next >= 0 && g_decode_trace_next < SVLM_TR_LAUNCHES && splits * b.kv_heads <= SVLM_TR_CTAS)
@@ -1232,13 +1264,13 @@ cudaError_t svlm_launch_decode(const SvlmAttendBatch& b, int layer0, int n_layer
             if (e != cudaSuccess) return e;
             cfg.dynamicSmemBytes = decode_layer_smem<128>();
             e = cudaLaunchKernelEx(&cfg, decode_layer_kernel<128>, b, layer0, Qp, q_pos, q_heads, Op, splits, Kn, Vn,
-                                   early_loads TRACE_ARG);
+                                   early_loads, (unsigned char*)tagged TRACE_ARG);
         } else {
             e = svlm_allow_smem<decode_layer_kernel<64>>(decode_layer_smem<64>());
             if (e != cudaSuccess) return e;
             cfg.dynamicSmemBytes = decode_layer_smem<64>();
             e = cudaLaunchKernelEx(&cfg, decode_layer_kernel<64>, b, layer0, Qp, q_pos, q_heads, Op, splits, Kn, Vn,
-                                   early_loads TRACE_ARG);
+                                   early_loads, (unsigned char*)tagged TRACE_ARG);
         }
     } else if (b.head_dim == 128) {
         e = svlm_allow_smem<decode_stream_kernel<128>>(decode_stream_smem<128>());

@@ -15,6 +15,7 @@ struct svlm_cache {
     int pending_n = 0;            // n of the latest metadata append (layers 1.. must match)
     bool configured_locked = false;
     unsigned wait_limit_host = 0;  // source buffer of svlm_debug_set_wait_limit's copy
+    unsigned char* decode_tagged = nullptr;   // per-layer decode kernel: epochs and tagged records (device memory)
     // What the latest enqueued operation was, for the decode step's early loads: a decode of one layer
     // may start reading its pages while the previous kernel still runs only if that kernel was a decode
     // of another layer of this cache (which writes neither the metadata nor this layer's pages).

@@ -44,8 +44,6 @@ void svlm_launch_attend_simple(const SvlmAttendBatch& b, int layer0, int n_layer
 
 // split-KV decode, n_q = 1 (svlm_decode.cu)
 size_t svlm_decode_ws_floats(int layers_in_launch, int kv_heads, int head_dim, int splits);
-// the words in front of the records (arrival counters and the like) for a cache of `layers` layers
-size_t svlm_decode_ws_head_floats(int layers, int kv_heads);
 int svlm_decode_splits(int n_pages, int kv_heads, int problems);
 // The kernel keeps the list of active pages in shared memory: caches with more pages take the general kernel.
 bool svlm_decode_supported(int n_pages);
@@ -53,9 +51,13 @@ bool svlm_decode_supported(int n_pages);
 // un-rotated) are written to the cache by this launch.  early_loads != 0: the caller vouches that no kernel
 // enqueued since the one before the previous launch on this stream wrote this cache's metadata or the pages of the
 // layers attended here, so the kernel may read them before the previous kernel has finished.
+// tagged: the cache's area of svlm_decode_tagged_bytes(kv_heads, head_dim, splits) bytes for a launch of one cache
+// and one layer (the per-layer kernel, whose splits hand their partial results over in tagged words); null, or
+// several problems in the launch: the streaming kernel with its arrival counters in the view's scratch.
 cudaError_t svlm_launch_decode(const SvlmAttendBatch& b, int layer0, int n_layers, const void* Q, const int* q_pos,
                                int q_heads, void* out, int splits, const void* Knew, const void* Vnew, int early_loads,
-                               cudaStream_t st);
+                               void* tagged, cudaStream_t st);
+size_t svlm_decode_tagged_bytes(int kv_heads, int head_dim, int splits);
 
 // Q/K/V projection with the append as its epilogue, head_dim 128 (svlm_qkv_sm100.cu).  tmX, tmW: host copies of
 // the CUtensorMap of X [n][hidden] (64 x 128 box) and W [(q_heads + 2 kv_heads) * 128][hidden] (64 x 256 box), 128-byte swizzle.

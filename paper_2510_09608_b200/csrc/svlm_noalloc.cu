@@ -63,9 +63,9 @@ extern "C" int svlm_attend_decode_noalloc(svlm_cache* c, int layer, const void* 
     if (!svlm_decode_supported(d.n_pages)) return SVLM_ERR_TOO_LARGE;   // more pages than the kernel's page list holds
 
     const int splits = svlm_decode_splits(d.n_pages, d.kv_heads, 1);
-    // the counter words of a cache of this many layers, then one layer's partials
-    const size_t head = svlm_decode_ws_head_floats(d.layers, d.kv_heads);
-    const size_t need = (head - svlm_decode_ws_head_floats(1, d.kv_heads) +
+    // counters for every (layer, kv head) of the cache, then one layer's partials
+    auto up4 = [](size_t x) { return (x + 3) & ~(size_t)3; };
+    const size_t need = (up4((size_t)d.layers * d.kv_heads) - up4((size_t)d.kv_heads) +
                          svlm_decode_ws_floats(1, d.kv_heads, d.head_dim, splits)) * sizeof(float);
     if (need > kScratchBytes) return SVLM_ERR_TOO_LARGE;
 
@@ -79,9 +79,8 @@ extern "C" int svlm_attend_decode_noalloc(svlm_cache* c, int layer, const void* 
     // let their next launch read early: forget the record.
     c->last_decode_layer = -1;
     if (rc == SVLM_OK) {
-        // counter words first in the scratch: zero when the kernel starts (for the per-layer kernel's pair of
-        // arrivals and start value, equal would do; zero is equal)
-        const size_t counter_bytes = head * sizeof(unsigned);
+        // counters first in the scratch: they must be zero when the kernel starts
+        const size_t counter_bytes = (size_t)d.layers * d.kv_heads * sizeof(unsigned);
         if (cudaMemsetAsync(scratch, 0, counter_bytes, c->stream) != cudaSuccess) rc = SVLM_ERR_CUDA;
     }
     if (rc == SVLM_OK) {
@@ -95,7 +94,7 @@ extern "C" int svlm_attend_decode_noalloc(svlm_cache* c, int layer, const void* 
         b.rope_tab = d.rope_tab;
         b.q_varlen = 0;
         v.ws = scratch;
-        if (svlm_launch_decode(b, layer, 1, Q, q_pos, q_heads, out, splits, nullptr, nullptr, 0, c->stream) != cudaSuccess)
+        if (svlm_launch_decode(b, layer, 1, Q, q_pos, q_heads, out, splits, nullptr, nullptr, 0, nullptr, c->stream) != cudaSuccess)
             rc = SVLM_ERR_CUDA;
     }
     if (prev != c->device) cudaSetDevice(prev);

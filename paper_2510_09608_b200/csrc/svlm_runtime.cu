@@ -223,7 +223,7 @@ int attend_common(svlm_cache* const* caches, int n_caches, int layer, const void
     if (n_q == 1 && group <= 8 && svlm_decode_supported(c0->dev.n_pages)) {
         // split-KV decode; every cache's scratch was sized for this launch shape at creation
         const int splits = svlm_decode_splits(c0->dev.n_pages, c0->dev.kv_heads, n_caches * n_layers);
-        SVLM_CUDA(svlm_launch_decode(b, layer0, n_layers, Q, q_pos, q_heads, out, splits, Knew, Vnew, early, c0->stream));
+        SVLM_CUDA(svlm_launch_decode(b, layer0, n_layers, Q, q_pos, q_heads, out, splits, Knew, Vnew, early, c0->decode_tagged, c0->stream));
         return SVLM_OK;
     }
     if (Knew) return SVLM_ERR_ARG;   // the fused step exists for the split-KV kernel only
@@ -287,6 +287,8 @@ int svlm_cache_create(svlm_cache** out, int layers, int kv_heads, int head_dim, 
         const size_t one = svlm_decode_ws_floats(layers, kv_heads, head_dim, svlm_decode_splits(d.n_pages, kv_heads, 1));
         const size_t all = svlm_decode_ws_floats(layers, kv_heads, head_dim, svlm_decode_splits(d.n_pages, kv_heads, layers));
         A(dev_alloc(c, &d.ws, std::max(one, all)));
+        // the per-layer kernel's tagged records: zero-filled here, afterwards written by that kernel alone
+        A(dev_alloc(c, &c->decode_tagged, svlm_decode_tagged_bytes(kv_heads, head_dim, svlm_decode_splits(d.n_pages, kv_heads, 1))));
     }
     A(dev_alloc(c, &d.K, slab));
     A(dev_alloc(c, &d.V, slab));

@@ -81,11 +81,12 @@ def test_batched_decode_gives_up_counter_returns_to_zero():
             assert_close(s._stats(out[i], s.ref.attend(0, s.stream.q(0, s.last[0]), s.last[2])))
 
 
-def test_layer_decode_waiting_combiners_give_up_counter_returns_to_zero():
-    """The per-layer split-KV kernel (one cache, one layer): its copies are cp.async and cannot time out, but the last
-    few CTAs to arrive share the final combine and all but the very last of them poll the arrival counter.  With the
-    limit at 0 they give up before their first poll: time-out recorded, their shares of the output unwritten, and the
-    counter (arrivals and finished waiters in its two halves) back at zero whichever CTA completed it."""
+def test_layer_decode_combiners_give_up_and_the_next_launch_is_right():
+    """The per-layer split-KV kernel (one cache, one layer): its copies are cp.async and cannot time out, but the first
+    splits of a KV head combine all the splits' records and read a record's words again until they carry the launch's
+    tag.  With the limit at 0 they give up before a first try: time-out recorded, their shares of the output
+    undefined; the KV head's epoch moves on all the same, so that with the limit restored the next launches look for
+    fresh tags and combine correctly."""
     from harness import assert_close, bits_to_dev, dev_to_f64
     from paper_2510_09608_b200 import binding
     wl = _small(True)

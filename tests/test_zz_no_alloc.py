@@ -60,11 +60,10 @@ def test_noalloc_decode_matches_regular_entry_point_twice():
 
 
 def _scratch_need(layers, kv_heads, head_dim, splits):
-    """Bytes of the library's fixed array a call needs: one 4-byte arrival counter per (layer, KV head) and two more
-    words per KV head, rounded up to 16 bytes, then per (KV head, split) one record of 8 x head_dim bf16 partial
-    outputs + 8 maxima + 8 sums."""
+    """Bytes of the library's fixed array a call needs: one 4-byte arrival counter per (layer, KV head), rounded up
+    to 16 bytes, then per (KV head, split) one record of 8 x head_dim bf16 partial outputs + 8 maxima + 8 sums."""
     up4 = lambda x: (x + 3) // 4 * 4  # noqa: E731
-    return up4(layers * kv_heads + 2 * kv_heads) * 4 + kv_heads * splits * (16 * head_dim + 64)
+    return up4(layers * kv_heads) * 4 + kv_heads * splits * (16 * head_dim + 64)
 
 
 def test_noalloc_limit_both_sides():
