@@ -948,15 +948,35 @@ decode_layer_kernel(SvlmAttendBatch b, int layer, const uint16_t* __restrict__ Q
             cp_async_commit();
         };
         Units u;
+        // the value units that have to wait for a key slot go towards L2 meanwhile
+        auto value_to_l2 = [&](int row) {
+            for (int o = lane * 128; o < ITEM_BYTES; o += 32 * 128)
+                asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char*>(Vh + (size_t)row * D) + o));
+        };
         if (n_rounds > 0) {
             get_units(0, u);
-            issue_front(u);
-            // the value units that have to wait for a key slot: towards L2 meanwhile
+            if (early_loads) {
+                // Reading ahead of the previous kernel there is time, and that kernel's short dependent loads
+                // (query, partial results) queue behind whatever the whole grid has in flight: the warp asks
+                // for one unit's worth at a time (keys of unit j with the values of unit j, copied or
+                // prefetched) and lets it land before the next, a third of the burst's depth.
 #pragma unroll
-            for (int j = 1; j < UPW; ++j)
-                if (u.row[j] >= 0)
-                    for (int o = lane * 128; o < ITEM_BYTES; o += 32 * 128)
-                        asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char*>(Vh + (size_t)u.row[j] * D) + o));
+                for (int j = 0; j < UPW; ++j) {
+                    if (u.row[j] >= 0) {
+                        load_unit(Kh, u.row[j], my + j * ITEM_BYTES);
+                        if (j == 0) load_unit(Vh, u.row[0], my + UPW * ITEM_BYTES);
+                        else value_to_l2(u.row[j]);
+                    }
+                    cp_async_commit();
+                    if (j + 1 < UPW) cp_async_wait<0>();
+                }
+                cp_async_commit();   // (empty: the round's "all but the latest group" then covers the last keys)
+            } else {
+                issue_front(u);
+#pragma unroll
+                for (int j = 1; j < UPW; ++j)
+                    if (u.row[j] >= 0) value_to_l2(u.row[j]);
+            }
         }
         if (threadIdx.x == 0) STAMP(2);              // the first round's copies are issued
 
