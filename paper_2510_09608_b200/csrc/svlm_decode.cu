@@ -955,8 +955,8 @@ decode_layer_kernel(SvlmAttendBatch b, int layer, const uint16_t* __restrict__ Q
         };
         if (n_rounds > 0) {
             get_units(0, u);
-            if (early_loads) {
-                // Reading ahead of the previous kernel there is time, and that kernel's short dependent loads
+            if (early_loads == 2) {
+                // Reading ahead of a previous decode step there is time, and that kernel's short dependent loads
                 // (query, partial results) queue behind whatever the whole grid has in flight: the warp asks
                 // for one unit's worth at a time (keys of unit j with the values of unit j, copied or
                 // prefetched) and lets it land before the next, a third of the burst's depth.

@@ -20,6 +20,7 @@ struct svlm_cache {
     // may start reading its pages while the previous kernel still runs only if that kernel was a decode
     // of another layer of this cache (which writes neither the metadata nor this layer's pages).
     int last_decode_layer = -1;   // layer of the latest operation if it was a single-layer decode, else -1
+    int calls_since_decode = 0;   // library calls on this cache's stream since that decode that left the record alone (projections)
     int last_decode_batch = 0;    // how many caches that launch served, and the first of them
     const svlm_cache* last_decode_first = nullptr;
     SvlmCacheDev* dev_copy = nullptr;   // `dev` in device memory, for the batched kernels

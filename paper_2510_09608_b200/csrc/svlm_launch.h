@@ -51,6 +51,8 @@ bool svlm_decode_supported(int n_pages);
 // un-rotated) are written to the cache by this launch.  early_loads != 0: the caller vouches that no kernel
 // enqueued since the one before the previous launch on this stream wrote this cache's metadata or the pages of the
 // layers attended here, so the kernel may read them before the previous kernel has finished.
+// early_loads == 2: moreover that previous kernel was itself a decode step of this cache (the per-layer kernel then
+// paces its read-ahead, one unit's worth per warp at a time).
 // tagged: the cache's area of svlm_decode_tagged_bytes(kv_heads, head_dim, splits) bytes for a launch of one cache
 // and one layer (the per-layer kernel, whose splits hand their partial results over in tagged words); null, or
 // several problems in the launch: the streaming kernel with its arrival counters in the view's scratch.

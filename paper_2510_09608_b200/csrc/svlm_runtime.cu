@@ -212,10 +212,14 @@ int attend_common(svlm_cache* const* caches, int n_caches, int layer, const void
                 c->last_decode_first != c0 || c->stream != c0->stream)
                 early = 0;
         }
+        // 2: nothing but that decode ran since (a chain of decode steps): the read-ahead has a whole layer-step of
+        // time and is paced; 1: other kernels ran in between (projections): read ahead at once
+        if (early && c0->calls_since_decode == 0) early = 2;
         for (int i = 0; i < n_caches; ++i) {
             caches[i]->last_decode_layer = layer;
             caches[i]->last_decode_batch = n_caches;
             caches[i]->last_decode_first = c0;
+            caches[i]->calls_since_decode = 0;
         }
     } else {
         for (int i = 0; i < n_caches; ++i) caches[i]->last_decode_layer = -1;
@@ -427,7 +431,9 @@ int svlm_out_proj(svlm_cache* c, const void* A, const void* Wo, int in_dim, int 
     if (((uintptr_t)A | (uintptr_t)Wo | (uintptr_t)Y) & 15) return SVLM_ERR_ARG;
     DeviceGuard guard(c->device);
     // The cache's record of its latest decode launch stays as it is: this call neither reads nor writes the
-    // cache, so a decode step that follows may still fetch its pages early.
+    // cache, so a decode step that follows may still fetch its pages early.  It does remember that something ran in
+    // between: the decode then has less time before its inputs are ready and does not pace its read-ahead.
+    ++c->calls_since_decode;
     if (svlm_gemv_supported(n, in_dim)) {      // a few tokens (decode): reading Wo once is all the work
         SVLM_CUDA(svlm_launch_gemv(A, Wo, Y, n, in_dim, out_dim, c->stream));
         return SVLM_OK;
