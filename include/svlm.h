@@ -256,7 +256,9 @@ int svlm_decode_step_host(svlm_cache* c, int layer, const void* K_host, const vo
  *   - the first call on each GPU looks up the array's device address, which can load the library's
  *     code on that GPU: make that first call before starting any stream capture.
  * Errors: SVLM_ERR_ARG, SVLM_ERR_ORDER (nothing appended yet), SVLM_ERR_TOO_LARGE, SVLM_ERR_CUDA.
- * The result equals svlm_attend's for the same state and inputs.
+ * The result agrees with svlm_attend's for the same state and inputs to within the rounding of the bf16
+ * partial results (the streaming split-KV kernel computes it; svlm_attend serves one layer of one
+ * cache with a kernel that keeps its partial results in a cache-owned area).
  */
 #define SVLM_NOALLOC_SCRATCH_BYTES (512u << 10)
 int svlm_attend_decode_noalloc(svlm_cache* c, int layer, const void* Q, const int32_t* q_pos, int q_heads, void* out);

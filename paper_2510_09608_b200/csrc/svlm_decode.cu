@@ -392,7 +392,7 @@ __device__ __forceinline__ void combine_tagged(int share, int shares, int splits
 #pragma unroll
             for (int k = 0; k < 2; ++k) want[k] = valid && r0 + k * DEC_WARPS * 4 < splits;
             for (unsigned polls = 0;; ++polls) {
-                if (polls >= wait_limit) { timed_out = true; break; }
+                if (__builtin_expect(polls >= wait_limit, 0)) { timed_out = true; break; }
                 bool ok = true;
 #pragma unroll
                 for (int k = 0; k < 2; ++k) {
@@ -482,7 +482,7 @@ __device__ __forceinline__ void combine_tagged(int share, int shares, int splits
         if (g0 + 8 < per) __syncthreads();   // the slabs are read before the next round writes them
     }
     if (share == 0 && threadIdx.x == 0) __stcg(epoch, tag);
-    if (timed_out) atomicCAS(status, 0, -5);   // SVLM_ERR_TIMEOUT
+    if (__builtin_expect(timed_out, 0)) atomicCAS(status, 0, -5);   // SVLM_ERR_TIMEOUT
 }
 
 // =============================== streaming kernel (several problems per launch) ===============================
@@ -1054,7 +1054,7 @@ decode_layer_kernel(SvlmAttendBatch b, int layer, const uint16_t* __restrict__ Q
         const int new_row16 = new_slot & ~15;          // first slot of the unit that holds the new token (fused step)
 
         for (int r = 0; r < n_rounds; ++r) {
-            if (r > 0) {                               // (larger caches only) the previous round is consumed: load the next
+            if (__builtin_expect(r > 0, 0)) {          // (larger caches only) the previous round is consumed: load the next
                 __syncwarp();
                 get_units(r, u);
                 issue_front(u);
@@ -1068,7 +1068,7 @@ decode_layer_kernel(SvlmAttendBatch b, int layer, const uint16_t* __restrict__ Q
 #pragma unroll
             for (int j = 0; j < UPW; ++j)
                 if (new_slot >= 0 && u.row[j] == new_row16) newj = j;
-            if (newj >= 0) {
+            if (__builtin_expect(newj >= 0, 0)) {
                 // fused append, key half: the rotated key goes into its shared-memory row and into the cache
                 uint16_t* kdst = const_cast<uint16_t*>(Kh) + (size_t)new_slot * D;
                 unsigned char* skw = my + newj * ITEM_BYTES;
@@ -1148,7 +1148,7 @@ decode_layer_kernel(SvlmAttendBatch b, int layer, const uint16_t* __restrict__ Q
                 pb[j][1] = movmatrix_trans(pack_bf16(p[2], p[3]));
             }
             if (threadIdx.x == 32 && r == 0) STAMP(14);  // warp 1: scores and softmax done
-            if (r > 0) {
+            if (__builtin_expect(r > 0, 0)) {
 #pragma unroll
                 for (int db = 0; db < DBLK; ++db) {
                     o[db][0] *= corr[0]; o[db][2] *= corr[0];
@@ -1162,7 +1162,7 @@ decode_layer_kernel(SvlmAttendBatch b, int layer, const uint16_t* __restrict__ Q
                 if (j == 1) cp_async_wait<0>();        // the two that followed the scores
                 if (j < 2) __syncwarp();
                 if (u.row[j] < 0) continue;
-                if (newj == j) {                       // fused append, value half
+                if (__builtin_expect(newj == j, 0)) {  // fused append, value half
                     uint16_t* vdst = const_cast<uint16_t*>(Vh) + (size_t)new_slot * D;
 #pragma unroll 1
                     for (int e2 = lane; e2 < D; e2 += 32) {

@@ -477,3 +477,57 @@ def test_per_layer_decode_with_several_rounds_per_cta(d):
             assert_close(s.attend(0))
             assert_close(s.attend(1))
     s.check_kv(1)
+
+
+@pytest.mark.parametrize("d", [64, 128])
+def test_per_layer_decode_many_launches_in_a_row(d):
+    """The per-layer decode kernel hands its splits' partial results over in words that carry the launch's tag (the KV
+    head's epoch + 1) and a launch trusts a word by its tag alone: several hundred launches on one cache, every one with
+    another query and a few of them replayed from a CUDA graph (where nothing on the host changes between launches), must
+    each give that query's result, never a word left by an earlier launch."""
+    from harness import SideBySide, assert_close, bits_to_dev, dev_to_f64
+    base = _wl(2) if d == 128 else _wl(1)
+    wl = dataclasses.replace(base, layers=2, q_heads=8, kv_heads=2, head_dim=d, n_sink=16, vision_window=5 * 128, text_window=100,
+                             frames=1, grid_h=8, grid_w=8, text_max=12, decode_steps=1)
+    s = SideBySide(wl)
+    for _ in range(6):
+        s.append_chunk()
+        s.evict()
+    s.append_decode_token()
+    gids, _, pos = s.last
+    qp = torch.from_numpy(np.ascontiguousarray(pos)).cuda()
+    rng = np.random.default_rng(11)
+    for l in range(wl.layers):
+        s._give_values_to_ref(l)
+    from oracle import qkv
+    Qs = [qkv.to_bf16_bits(rng.standard_normal((1, wl.q_heads, d))) for _ in range(6)]
+    Qd = [bits_to_dev(q) for q in Qs]
+    want = [[s.ref.attend(l, Qs[i], pos) for i in range(len(Qs))] for l in range(wl.layers)]
+    for it in range(240):
+        i, l = it % len(Qs), (it // 7) % wl.layers
+        out = s.cache.attend(l, Qd[i], qp)
+        if it % 17 == 0 or it >= 236:
+            assert_close(s._stats(dev_to_f64(out), want[l][i]))
+    # the same from a graph: six launches per replay, replayed five times, outputs in fixed buffers
+    outs = [torch.empty_like(Qd[0]) for _ in Qd]
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        s.cache.set_stream(side)
+        for i in range(len(Qd)):
+            s.cache.attend(i % wl.layers, Qd[i], qp, out=outs[i])      # warm-up outside the capture
+        side.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            for i in range(len(Qd)):
+                s.cache.attend(i % wl.layers, Qd[i], qp, out=outs[i])
+        for _ in range(5):
+            for o in outs:
+                o.zero_()
+            g.replay()
+            side.synchronize()
+            for i in range(len(Qd)):
+                assert_close(s._stats(dev_to_f64(outs[i]), want[i % wl.layers][i]))
+    torch.cuda.current_stream().wait_stream(side)
+    s.cache.set_stream(torch.cuda.current_stream())
+    assert s.cache.status() == 0
