@@ -227,7 +227,13 @@ int svlm_cache_append_host(svlm_cache* c, int layer, const void* K_host, const v
                            const uint8_t* token_type_host, const int32_t* pos_host, int n);
 int svlm_attend_host(svlm_cache* c, int layer, const void* Q_host, const int32_t* q_pos_host, int n_q, int q_heads,
                      void* out_host);
-/* svlm_decode_step with host buffers (layer -1: all layers of the token in one launch); returns with out_host filled. */
+/*
+ * svlm_decode_step with host buffers (layer -1: all layers of the token in one launch); returns with out_host
+ * filled.  The step's inputs are a few KB: they are gathered in a page-locked buffer of the library and go up in
+ * one copy.  For layer -1, when every buffer is itself page-locked and mapped (as pinned allocations are under
+ * unified addressing) and 16-byte aligned, nothing is copied at all: the kernels read the inputs and write the
+ * output where they are.
+ */
 int svlm_decode_step_host(svlm_cache* c, int layer, const void* K_host, const void* V_host, const uint8_t* token_type_host,
                           const int32_t* pos_host, const void* Q_host, int q_heads, void* out_host);
 

@@ -27,6 +27,8 @@ struct svlm_cache {
     // staging for the *_host entry points
     void* stage = nullptr;
     size_t stage_bytes = 0;
+    void* hstage = nullptr;       // page-locked host buffer: small inputs of a host-buffer call are gathered here for one copy
+    size_t hstage_bytes = 0;
     // copy streams and per-layer events of the pipelined host-buffer chunk prefill (created on first use)
     cudaStream_t copy_in = nullptr, copy_out = nullptr;
     cudaEvent_t ev_start = nullptr;

@@ -333,6 +333,24 @@ def test_host_buffer_entry_points_equal_the_device_ones():
                                       pin(Q.view(np.int16)), got)
             assert host.status() == binding.OK
             assert np.array_equal(got.numpy().view(np.uint16), want.view(torch.int16).cpu().numpy().view(np.uint16)), step
+        # a generated token layer by layer: pinned buffers (the kernels read them in place) and, every other step,
+        # pageable ones (staged through device memory) against the device-pointer calls
+        gids, types, pos = stream.next_decode_token()
+        ty, ps = torch.from_numpy(types), torch.from_numpy(np.ascontiguousarray(pos))
+        for l in range(wl.layers):
+            K, V, Q = stream.k(l, gids), stream.v(l, gids), stream.q(l, gids)
+            want = dev.decode_step(l, bits_to_dev(K), bits_to_dev(V), ty.cuda() if l == 0 else None, ps.cuda(), bits_to_dev(Q))
+            if step % 2:
+                got = np.zeros(Q.shape, dtype=np.uint16)
+                host.decode_step_host(l, np.ascontiguousarray(K), np.ascontiguousarray(V), types if l == 0 else None,
+                                      np.ascontiguousarray(pos), np.ascontiguousarray(Q), got)
+            else:
+                got_t = torch.zeros(Q.shape, dtype=torch.int16).pin_memory()
+                host.decode_step_host(l, pin(K.view(np.int16)), pin(V.view(np.int16)), ty.pin_memory() if l == 0 else None,
+                                      ps.pin_memory(), pin(Q.view(np.int16)), got_t)
+                got = got_t.numpy().view(np.uint16)
+            assert host.status() == binding.OK
+            assert np.array_equal(got, want.view(torch.int16).cpu().numpy().view(np.uint16)), (step, l)
     a, b = dev.query(), host.query()
     assert np.array_equal(a["gids"], b["gids"]) and np.array_equal(a["pos"], b["pos"])
 
